@@ -1,0 +1,129 @@
+/*
+ * rabit.h -- C ABI of the B200 residual-binary linear layer library.
+ *
+ * The layer (paper Section 4.1 and Eq. 2, "stacked binary weight") is
+ *
+ *     y[b][i] = sum_{k<K} g_k[i] * sum_{j<N} B_k[i][j] * h_k[j] * x[b][j]
+ *
+ * with K stacked sign matrices B_k in {-1,+1}^{M x N}, a per-output scale g_k (length M)
+ * and a per-input scale h_k (length N) per path; at inference the sign matrices are frozen
+ * and only bits + scales remain (end of Section 4.2).  Signs are stored one bit each,
+ * +1 -> 0 and -1 -> 1 (Appendix "Weight Packing").
+ *
+ * Conventions
+ *   - M = d_out, N = d_in, K = number of paths (1..3), batch = number of activation rows.
+ *   - Every function returns RABIT_OK (0) or a negative rabit_status; none throws, prints
+ *     or exits.  rabit_last_error() returns a thread-local description of the last failure.
+ *   - "HOST" / "DEVICE" on a pointer says which memory it must point into.
+ *   - Device memory is always owned by the caller (for example a torch tensor); the library
+ *     never frees it.  A rabit_layer is a small host-side descriptor that refers to it.
+ *   - All device work is enqueued on the cudaStream_t passed as `stream` (void*, may be 0).
+ */
+#ifndef RABIT_H_
+#define RABIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RABIT_API __attribute__((visibility("default")))
+#else
+#define RABIT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum rabit_status {
+    RABIT_OK = 0,
+    RABIT_INVALID_ARG = -1,        /* null pointer, misaligned pointer, aliasing, batch < 1 ... */
+    RABIT_UNSUPPORTED_SHAPE = -2,  /* K outside 1..3, M < 1, N < 32 or N not a multiple of 32 */
+    RABIT_BUFFER_TOO_SMALL = -3,   /* dev_bytes / out_bytes below the required size */
+    RABIT_CUDA_ERROR = -4,         /* a CUDA runtime call failed; see rabit_last_error() */
+    RABIT_DEVICE_FAULT = -5        /* a kernel reported an internal bounded wait that ran out */
+} rabit_status;
+
+typedef struct rabit_layer rabit_layer;   /* opaque host-side descriptor */
+
+/* Version of the packed device layout written by rabit_pack_host (also stored in its header). */
+RABIT_API int rabit_layout_version(void);
+
+/*
+ * Bytes of the packed image of a K x M x N layer: header + interleaved sign tiles + padded
+ * fp16 scales + the per-layer reduction scratch.  Returns 0 for an unsupported shape.
+ * (Storage accounting of Section 4.1: K bits per weight plus the scale vectors.)
+ */
+RABIT_API size_t rabit_packed_bytes(int K, int M, int N);
+
+/*
+ * Step "pack" (Appendix "Weight Packing", re-designed layout): permute canonical sign planes
+ * and scales into the device layout, entirely on the host.
+ *   planes  HOST  uint32 [K][M][N/32]; column j is bit (j % 32), LSB first, of word j / 32;
+ *                 bit 1 means -1, bit 0 means +1.
+ *   g       HOST  fp16 bit patterns [K][M]   (per-output scale of each path)
+ *   h       HOST  fp16 bit patterns [K][N]   (per-input scale of each path)
+ *   out     HOST  receives rabit_packed_bytes(K,M,N) bytes; out_bytes must be at least that.
+ * Needs no GPU.  The image is byte-for-byte what rabit_pack places in device memory.
+ */
+RABIT_API int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
+                    int K, int M, int N, void* out, size_t out_bytes);
+
+/*
+ * Inverse of rabit_pack_host on a HOST image: recovers canonical planes and scales
+ * bit-exactly.  Any of planes_out / g_out / h_out may be NULL to skip it.
+ */
+RABIT_API int rabit_unpack_host(const void* image, size_t image_bytes,
+                      uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out);
+
+/*
+ * Pack (as rabit_pack_host) and copy the image into caller-owned device memory, then create
+ * the descriptor.
+ *   dev_buf   DEVICE  256-byte aligned, dev_bytes >= rabit_packed_bytes(K,M,N); must stay
+ *                     valid and unmodified by the caller until rabit_free.
+ *   stream    the copy is enqueued on it and the call returns after it has completed.
+ *   out       receives the new descriptor.
+ * The reduction scratch inside dev_buf starts zeroed and is left zeroed by every call of
+ * rabit_linear, so calls on one layer must not overlap in time (different layers may).
+ */
+RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
+               int K, int M, int N, void* dev_buf, size_t dev_bytes, void* stream,
+               rabit_layer** out);
+
+/*
+ * Run the layer (Section 4.1 forward with the Eq. 2 weight):
+ *   x  DEVICE fp16 [batch][N] row-major, 16-byte aligned
+ *   y  DEVICE fp16 [batch][M] row-major, 16-byte aligned, must not overlap x
+ * Asynchronous on `stream`; allocates nothing, never synchronises, and may be captured in
+ * a CUDA graph.  batch <= 16 runs the bandwidth-bound GEMV family, larger batches the
+ * tensor-core GEMM.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end.
+ */
+RABIT_API int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
+
+/* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
+RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
+                 void* stream);
+
+/* Shape queries on a descriptor; return -1 on a NULL layer. */
+RABIT_API int rabit_layer_K(const rabit_layer* layer);
+RABIT_API int rabit_layer_M(const rabit_layer* layer);
+RABIT_API int rabit_layer_N(const rabit_layer* layer);
+
+/*
+ * Choose the kernel family for subsequent rabit_linear calls of this layer:
+ *   0 = automatic (default), 1 = plain sign-select kernel, 2 = integer tensor-core GEMV,
+ *   3 = tcgen05 GEMM.  Returns RABIT_INVALID_ARG for a variant that cannot run the layer.
+ * Meant for A/B timing and profiling; results are within tolerance for every variant.
+ */
+RABIT_API int rabit_set_variant(rabit_layer* layer, int variant);
+
+/* Release the descriptor only; the caller's device buffer is untouched. NULL is accepted. */
+RABIT_API int rabit_free(rabit_layer* layer);
+
+/* Thread-local, never NULL; empty string if the last call on this thread succeeded. */
+RABIT_API const char* rabit_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RABIT_H_ */

@@ -1,0 +1,198 @@
+"""ctypes binding of the C ABI in include/rabit.h.  Marshalling only: every step of the layer
+runs inside the CUDA library."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librabit.so")
+
+_c_void_p = ctypes.c_void_p
+_c_int = ctypes.c_int
+_c_size_t = ctypes.c_size_t
+
+
+class RabitError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"rabit error {code}: {message}")
+        self.code = code
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2602_05367_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    lib.rabit_layout_version.restype = _c_int
+    lib.rabit_packed_bytes.restype = _c_size_t
+    lib.rabit_packed_bytes.argtypes = [_c_int, _c_int, _c_int]
+    lib.rabit_pack_host.restype = _c_int
+    lib.rabit_pack_host.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_size_t]
+    lib.rabit_unpack_host.restype = _c_int
+    lib.rabit_unpack_host.argtypes = [_c_void_p, _c_size_t, _c_void_p, _c_void_p, _c_void_p]
+    lib.rabit_pack.restype = _c_int
+    lib.rabit_pack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_size_t,
+                               _c_void_p, ctypes.POINTER(_c_void_p)]
+    lib.rabit_linear.restype = _c_int
+    lib.rabit_linear.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
+    lib.rabit_unpack.restype = _c_int
+    lib.rabit_unpack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p]
+    for name in ("rabit_layer_K", "rabit_layer_M", "rabit_layer_N"):
+        getattr(lib, name).restype = _c_int
+        getattr(lib, name).argtypes = [_c_void_p]
+    lib.rabit_set_variant.restype = _c_int
+    lib.rabit_set_variant.argtypes = [_c_void_p, _c_int]
+    lib.rabit_free.restype = _c_int
+    lib.rabit_free.argtypes = [_c_void_p]
+    lib.rabit_last_error.restype = ctypes.c_char_p
+    if hasattr(lib, "rabit_linear_static_scratch"):
+        lib.rabit_linear_static_scratch.restype = _c_int
+        lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
+        lib.rabit_static_scratch_max_bytes.restype = _c_size_t
+    return lib
+
+
+_lib = _load()
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def raw_lib() -> ctypes.CDLL:
+    """The loaded CDLL, for tests that exercise the ABI with raw pointers."""
+    return _lib
+
+
+def last_error() -> str:
+    return _lib.rabit_last_error().decode()
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise RabitError(rc, last_error())
+
+
+def layout_version() -> int:
+    return int(_lib.rabit_layout_version())
+
+
+def packed_bytes(K: int, M: int, N: int) -> int:
+    return int(_lib.rabit_packed_bytes(K, M, N))
+
+
+def _host_arrays(planes, g, h) -> Tuple[np.ndarray, np.ndarray, np.ndarray, int, int, int]:
+    planes = np.ascontiguousarray(planes, dtype=np.uint32)
+    g16 = np.ascontiguousarray(g, dtype=np.float16).view(np.uint16)
+    h16 = np.ascontiguousarray(h, dtype=np.float16).view(np.uint16)
+    if planes.ndim != 3 or g16.ndim != 2 or h16.ndim != 2:
+        raise ValueError("planes must be [K][M][N/32], g [K][M], h [K][N]")
+    K, M, W = planes.shape
+    N = h16.shape[1]
+    if g16.shape != (K, M) or h16.shape[0] != K or W * 32 != N:
+        raise ValueError("inconsistent shapes between planes, g and h")
+    return planes, g16, h16, K, M, N
+
+
+def pack_host(planes, g, h) -> np.ndarray:
+    """Packed image as a uint8 array (no GPU needed)."""
+    planes, g16, h16, K, M, N = _host_arrays(planes, g, h)
+    nbytes = packed_bytes(K, M, N)
+    if nbytes == 0:
+        raise RabitError(-2, f"unsupported shape K={K} M={M} N={N}")
+    out = np.empty(nbytes, dtype=np.uint8)
+    _check(_lib.rabit_pack_host(planes.ctypes.data, g16.ctypes.data, h16.ctypes.data, K, M, N,
+                                out.ctypes.data, out.nbytes))
+    return out
+
+
+def unpack_host(image: np.ndarray, K: int, M: int, N: int):
+    image = np.ascontiguousarray(image, dtype=np.uint8)
+    planes = np.empty((K, M, N // 32), dtype=np.uint32)
+    g = np.empty((K, M), dtype=np.uint16)
+    h = np.empty((K, N), dtype=np.uint16)
+    _check(_lib.rabit_unpack_host(image.ctypes.data, image.nbytes, planes.ctypes.data, g.ctypes.data, h.ctypes.data))
+    return planes, g.view(np.float16), h.view(np.float16)
+
+
+class RabitLayer:
+    """Owns one descriptor and the torch buffer that holds its packed image."""
+
+    def __init__(self, handle: int, dev_buf, K: int, M: int, N: int):
+        self._handle = _c_void_p(handle)
+        self.dev_buf = dev_buf          # keeps the device memory alive
+        self.K, self.M, self.N = K, M, N
+
+    @property
+    def handle(self) -> ctypes.c_void_p:
+        if self._handle is None:
+            raise RabitError(-1, "layer already freed")
+        return self._handle
+
+    def set_variant(self, variant: int) -> None:
+        _check(_lib.rabit_set_variant(self.handle, variant))
+
+    def unpack(self, stream: int = 0):
+        planes = np.empty((self.K, self.M, self.N // 32), dtype=np.uint32)
+        g = np.empty((self.K, self.M), dtype=np.uint16)
+        h = np.empty((self.K, self.N), dtype=np.uint16)
+        _check(_lib.rabit_unpack(self.handle, planes.ctypes.data, g.ctypes.data, h.ctypes.data, _c_void_p(stream)))
+        return planes, g.view(np.float16), h.view(np.float16)
+
+    def free(self) -> None:
+        if self._handle is not None:
+            _lib.rabit_free(self._handle)
+            self._handle = None
+            self.dev_buf = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def rabit_pack(planes, g, h, device="cuda:0", stream: Optional[int] = None) -> RabitLayer:
+    """Pack on the host, upload into a torch-allocated device buffer, return the layer."""
+    import torch
+
+    planes, g16, h16, K, M, N = _host_arrays(planes, g, h)
+    nbytes = packed_bytes(K, M, N)
+    if nbytes == 0:
+        raise RabitError(-2, f"unsupported shape K={K} M={M} N={N}")
+    dev = torch.device(device)
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream(dev).cuda_stream if stream is None else stream
+    out = _c_void_p()
+    with torch.cuda.device(dev):
+        _check(_lib.rabit_pack(planes.ctypes.data, g16.ctypes.data, h16.ctypes.data, K, M, N,
+                               _c_void_p(buf.data_ptr()), nbytes, _c_void_p(st), ctypes.byref(out)))
+    return RabitLayer(out.value, buf, K, M, N)
+
+
+def rabit_linear(layer: RabitLayer, x, y=None, stream: Optional[int] = None):
+    """y[b] = layer(x[b]); x is a CUDA fp16 tensor [batch][N] (or [N]); returns y [batch][M]."""
+    import torch
+
+    if x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA float16 tensor")
+    xb = x if x.dim() == 2 else x.view(1, -1)
+    if xb.shape[1] != layer.N:
+        raise ValueError(f"x has {xb.shape[1]} columns, layer expects {layer.N}")
+    batch = xb.shape[0]
+    if y is None:
+        y = torch.empty((batch, layer.M), dtype=torch.float16, device=x.device)
+    elif y.dtype != torch.float16 or not y.is_cuda or not y.is_contiguous() or y.numel() != batch * layer.M:
+        raise ValueError("y must be a contiguous CUDA float16 tensor of batch*M elements")
+    st = torch.cuda.current_stream(x.device).cuda_stream if stream is None else stream
+    _check(_lib.rabit_linear(layer.handle, _c_void_p(xb.data_ptr()), _c_void_p(y.data_ptr()), batch, _c_void_p(st)))
+    return y if x.dim() == 2 else y.view(-1)
+
+
+def rabit_free(layer: RabitLayer) -> None:
+    layer.free()

@@ -1,0 +1,149 @@
+// C ABI of the library: argument checks, pack/upload, dispatch, error strings.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "rabit_internal.h"
+
+static thread_local char g_err[512] = {0};
+
+int rabit_fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+void rabit_clear_error() { g_err[0] = 0; }
+
+extern "C" const char* rabit_last_error(void) { return g_err; }
+
+extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
+                          int K, int M, int N, void* dev_buf, size_t dev_bytes, void* stream,
+                          rabit_layer** out) {
+    rabit_clear_error();
+    if (!out) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: out is NULL");
+    *out = nullptr;
+    if (!planes || !g || !h || !dev_buf) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: null pointer");
+    if (((uintptr_t)dev_buf & 255u) != 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: dev_buf must be 256-byte aligned");
+    RabitGeom G;
+    if (!rabit_make_geom(K, M, N, &G))
+        return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_pack: unsupported shape K=%d M=%d N=%d (need 1<=K<=3, M>=1, N%%32==0)", K, M, N);
+    RabitHeader hdr;
+    rabit_fill_header(G, &hdr);
+    if (dev_bytes < hdr.total_bytes)
+        return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_pack: dev_buf holds %zu bytes, layer needs %zu", dev_bytes, (size_t)hdr.total_bytes);
+
+    cudaPointerAttributes attr;
+    RABIT_CUDA_TRY(cudaPointerGetAttributes(&attr, dev_buf));
+    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: dev_buf is not device memory");
+
+    std::vector<uint8_t> image;
+    try {
+        image.resize(hdr.total_bytes);
+    } catch (const std::bad_alloc&) {
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: out of host memory for the staging image");
+    }
+    int rc = rabit_pack_host(planes, g, h, K, M, N, image.data(), image.size());
+    if (rc != RABIT_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(dev_buf, image.data(), hdr.total_bytes, cudaMemcpyHostToDevice, st));
+    RABIT_CUDA_TRY(cudaStreamSynchronize(st));
+
+    rabit_layer* L = new (std::nothrow) rabit_layer;
+    if (!L) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: out of host memory");
+    L->geom = G;
+    L->device = attr.device;
+    L->variant = 0;
+    L->sm_count = 0;
+    cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, attr.device);
+    L->dev_base = (char*)dev_buf;
+    L->dev_bytes = hdr.total_bytes;
+    L->d_bits = (const uint4*)(L->dev_base + hdr.off_bits);
+    L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
+    L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
+    L->d_partial = (float*)(L->dev_base + hdr.off_partial);
+    L->d_counters = (unsigned int*)(L->dev_base + hdr.off_counters);
+    *out = L;
+    return RABIT_OK;
+}
+
+static bool ranges_overlap(const void* a, size_t an, const void* b, size_t bn) {
+    uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bn && b0 < a0 + an;
+}
+
+extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: layer is NULL");
+    if (!x || !y) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: null x or y");
+    if (batch < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: batch must be >= 1 (got %d)", batch);
+    if ((((uintptr_t)x) & 15u) || (((uintptr_t)y) & 15u))
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: x and y must be 16-byte aligned");
+    const RabitGeom& G = layer->geom;
+    if (ranges_overlap(x, (size_t)batch * G.N * 2, y, (size_t)batch * G.M * 2))
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: x and y overlap");
+    cudaStream_t st = (cudaStream_t)stream;
+
+    int variant = layer->variant;
+    if (variant == 0) {
+        if (batch <= RABIT_MAX_GEMV_BATCH)
+            variant = rabit_gemv_mma_supports(*layer, batch) ? 2 : 1;
+        else
+            variant = rabit_gemm_tc_supports(*layer, batch) ? 3 : 1;
+    }
+    cudaError_t e;
+    switch (variant) {
+        case 2:
+            if (!rabit_gemv_mma_supports(*layer, batch))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: integer-MMA GEMV cannot run batch %d", batch);
+            e = rabit_launch_gemv_mma(*layer, x, y, batch, st);
+            break;
+        case 3:
+            if (!rabit_gemm_tc_supports(*layer, batch))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: tcgen05 GEMM cannot run batch %d", batch);
+            e = rabit_launch_gemm_tc(*layer, x, y, batch, st);
+            break;
+        default:
+            e = rabit_launch_plain(*layer, x, y, batch, st);
+            break;
+    }
+    if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear: launch failed: %s", cudaGetErrorString(e));
+    return RABIT_OK;
+}
+
+extern "C" int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out, void* stream) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack: layer is NULL");
+    std::vector<uint8_t> image;
+    try {
+        image.resize(layer->dev_bytes);
+    } catch (const std::bad_alloc&) {
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack: out of host memory");
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(image.data(), layer->dev_base, layer->dev_bytes, cudaMemcpyDeviceToHost, st));
+    RABIT_CUDA_TRY(cudaStreamSynchronize(st));
+    return rabit_unpack_host(image.data(), image.size(), planes_out, g_out, h_out);
+}
+
+extern "C" int rabit_layer_K(const rabit_layer* layer) { return layer ? layer->geom.K : -1; }
+extern "C" int rabit_layer_M(const rabit_layer* layer) { return layer ? layer->geom.M : -1; }
+extern "C" int rabit_layer_N(const rabit_layer* layer) { return layer ? layer->geom.N : -1; }
+
+extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
+    if (variant < 0 || variant > 3) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..3");
+    layer->variant = variant;
+    return RABIT_OK;
+}
+
+extern "C" int rabit_free(rabit_layer* layer) {
+    rabit_clear_error();
+    delete layer;
+    return RABIT_OK;
+}

@@ -1,0 +1,47 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#ifndef RABIT_INTERNAL_H_
+#define RABIT_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/rabit.h"
+#include "rabit_layout.h"
+
+struct rabit_layer {
+    RabitGeom geom;
+    int device;
+    int variant;                 // 0 auto, 1 plain, 2 integer-MMA GEMV, 3 tcgen05 GEMM
+    int sm_count;
+    char* dev_base;              // caller-owned packed image
+    size_t dev_bytes;
+    const uint4* d_bits;         // sign tiles
+    const uint16_t* d_g;         // fp16 [K][Mp]
+    const uint16_t* d_h;         // fp16 [K][Np]
+    float* d_partial;            // fp32 [n_slices][Mp] reduction scratch (kept zero between calls)
+    unsigned int* d_counters;    // u32 [n_rt] arrival counters (kept zero between calls)
+};
+
+// error reporting (thread-local message); returns `code`
+int rabit_fail(int code, const char* fmt, ...);
+void rabit_clear_error();
+#define RABIT_CUDA_TRY(expr)                                                              \
+    do {                                                                                  \
+        cudaError_t e__ = (expr);                                                         \
+        if (e__ != cudaSuccess)                                                           \
+            return rabit_fail(RABIT_CUDA_ERROR, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+// geometry / layout (rabit_pack.cu)
+bool rabit_make_geom(int K, int M, int N, RabitGeom* out);
+void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr);
+
+// kernel launchers; each enqueues on `stream` and returns a cudaError_t from the launch
+cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+bool rabit_gemv_mma_supports(const rabit_layer& L, int batch);
+cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+bool rabit_gemm_tc_supports(const rabit_layer& L, int batch);
+
+#endif  // RABIT_INTERNAL_H_

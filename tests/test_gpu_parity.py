@@ -1,0 +1,147 @@
+"""GPU parity: the CUDA library (through the C ABI) against the float64 CPU oracle on
+identical seeded inputs, element by element, within
+    max_i |y_gpu - y_ref| <= 2e-3 * max_i sum_j sum_k |g_ki h_kj x_j| + 1e-5   per batch row."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import rabit_oracle as orc
+from synth import make_layer, make_x, make_planes_constant
+from tests.gpu_util import run_layer, check_against_oracle
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [0, 1]   # automatic, plain sign-select
+
+SMALL = [  # several tiles plus ragged tails in both dimensions
+    (2, 32, 128), (2, 100, 160), (2, 256, 1184), (3, 96, 640), (1, 33, 96), (2, 160, 2080), (2, 1000, 512),
+]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("K,M,N", SMALL)
+@pytest.mark.parametrize("batch", [1, 2])
+def test_small_shapes(K, M, N, batch, variant):
+    L = make_layer(M, N, K, key=(70, K, M, N))
+    x = make_x(batch, N, key=(70, M, N, batch))
+    y = run_layer(L, x, variant)
+    check_against_oracle(L, x, y)
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("batch", [3, 4, 5, 8, 16, 17, 40])
+def test_batches(batch, variant):
+    L = make_layer(192, 896, 2, key=(71,))
+    x = make_x(batch, 896, key=(71, batch))
+    y = run_layer(L, x, variant)
+    check_against_oracle(L, x, y)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_config0_full_size(variant):
+    """4096 x 4096, K=2, batch 1, seed 0 -- every output compared."""
+    L = make_layer(4096, 4096, 2, key=(0, 0, 0))
+    x = make_x(1, 4096, key=(0, 0))
+    y = run_layer(L, x, variant)
+    err, tol = check_against_oracle(L, x, y)
+    assert tol[0] > 0.1 and err[0] < tol[0]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_structured_inputs(variant):
+    K, M, N = 2, 96, 384
+    L = make_layer(M, N, K, key=(72,))
+    # unit vectors read single columns (bit order / layout permutation)
+    for j in [0, 1, 31, 32, 127, 128, 200, 383]:
+        x = np.zeros((1, N), dtype=np.float16); x[0, j] = 1.0
+        check_against_oracle(L, x, run_layer(L, x, variant))
+    # constant planes
+    for bit in (0, 1):
+        L.planes = make_planes_constant(K, M, N, bit)
+        x = make_x(1, N, key=(72, bit))
+        check_against_oracle(L, x, run_layer(L, x, variant))
+    # zero activations give exactly zero
+    L = make_layer(M, N, K, key=(72, 9))
+    y = run_layer(L, np.zeros((2, N), dtype=np.float16), variant)
+    assert not y.any()
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_outlier_activations(variant):
+    """A few huge activations among small ones (the dynamic range of real hidden states)."""
+    K, M, N = 2, 128, 2048
+    L = make_layer(M, N, K, key=(73,))
+    x = (make_x(2, N, key=(73,)).astype(np.float32) * 0.02)
+    x[0, 5] = 900.0; x[0, 1033] = -650.0; x[1, 77] = 1200.0
+    x = x.astype(np.float16)
+    check_against_oracle(L, x, run_layer(L, x, variant))
+
+
+def test_device_round_trip():
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(100, 288, 2, key=(74,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    planes, g, h = layer.unpack()
+    assert np.array_equal(planes, L.planes)
+    assert np.array_equal(g.view(np.uint16), L.g.view(np.uint16))
+    assert np.array_equal(h.view(np.uint16), L.h.view(np.uint16))
+    layer.free()
+
+
+def test_graph_capture_and_replay():
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(256, 512, 2, key=(75,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    x = torch.zeros((1, 512), dtype=torch.float16, device="cuda:0")
+    y = torch.empty((1, 256), dtype=torch.float16, device="cuda:0")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        rabit.rabit_linear(layer, x, y)        # warm-up outside capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            rabit.rabit_linear(layer, x, y)
+    for t in range(3):
+        xn = make_x(1, 512, key=(75, t))
+        x.copy_(torch.from_numpy(xn))
+        graph.replay()
+        torch.cuda.synchronize()
+        check_against_oracle(L, xn, y.cpu().numpy())
+    layer.free()
+
+
+def test_repeated_calls_leave_scratch_clean():
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(320, 1536, 2, key=(76,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    for t in range(4):
+        xn = make_x(2, 1536, key=(76, t))
+        y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
+        torch.cuda.synchronize()
+        check_against_oracle(L, xn, y.cpu().numpy())
+    layer.free()
+
+
+def test_argument_errors_on_device():
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from paper_2602_05367_b200 import binding
+    lib = binding.raw_lib()
+    L = make_layer(64, 128, 2, key=(77,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    buf = torch.zeros(4096, dtype=torch.float16, device="cuda:0")
+    p = buf.data_ptr()
+    vp = ctypes.c_void_p
+    assert lib.rabit_linear(layer.handle, vp(p + 2), vp(p + 2048), 1, None) == -1      # misaligned x
+    assert "aligned" in rabit.last_error()
+    assert lib.rabit_linear(layer.handle, vp(p), vp(p + 128), 1, None) == -1           # y overlaps x
+    assert lib.rabit_linear(layer.handle, vp(p), vp(p + 2048), 0, None) == -1          # batch < 1
+    host = np.zeros(rabit.packed_bytes(2, 64, 128), dtype=np.uint8)
+    out = vp()
+    rc = lib.rabit_pack(L.planes.ctypes.data, L.g.view(np.uint16).ctypes.data, L.h.view(np.uint16).ctypes.data,
+                        2, 64, 128, vp(p), 16, None, ctypes.byref(out))
+    assert rc == -3                                                                     # device buffer too small
+    layer.free()

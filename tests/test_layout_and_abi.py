@@ -1,0 +1,121 @@
+"""CPU-side tests of the product's host logic: the packed layout (bit-exact against the
+reference statement of the format), its round trip, argument checking, and that the C-ABI
+library exports every symbol the header declares.  No GPU is touched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2602_05367_b200 as rabit
+from paper_2602_05367_b200 import binding
+from oracle import layout_spec as spec
+from synth import make_layer, make_planes_constant
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+SHAPES = [(1, 32, 32), (2, 32, 128), (2, 64, 256), (2, 100, 160), (3, 33, 1056), (2, 160, 640), (1, 7, 96),
+          (2, 256, 1184)]
+
+
+@pytest.mark.parametrize("K,M,N", SHAPES)
+def test_library_image_equals_spec(K, M, N):
+    L = make_layer(M, N, K, key=(80, K, M, N))
+    img = rabit.pack_host(L.planes, L.g, L.h)
+    hd = spec.read_header(img)
+    assert hd["magic"] == spec.MAGIC and hd["version"] == rabit.layout_version() == spec.VERSION
+    want = spec.pack_spec(L.planes, L.g, L.h, hd["slice_cg"])
+    assert img.nbytes == want.nbytes == rabit.packed_bytes(K, M, N)
+    assert np.array_equal(img, want)
+
+
+@pytest.mark.parametrize("K,M,N", SHAPES)
+def test_round_trip_bit_exact(K, M, N):
+    L = make_layer(M, N, K, key=(81, K, M, N))
+    img = rabit.pack_host(L.planes, L.g, L.h)
+    planes, g, h = rabit.unpack_host(img, K, M, N)
+    assert np.array_equal(planes, L.planes)
+    assert np.array_equal(g.view(np.uint16), L.g.view(np.uint16))
+    assert np.array_equal(h.view(np.uint16), L.h.view(np.uint16))
+    # the reference unpacker reads the library image the same way
+    if M * N <= 64 * 256:
+        p2, g2, h2 = spec.unpack_spec(img)
+        assert np.array_equal(p2, L.planes) and np.array_equal(g2.view(np.uint16), L.g.view(np.uint16))
+        assert np.array_equal(h2.view(np.uint16), L.h.view(np.uint16))
+
+
+@pytest.mark.parametrize("slice_cg", [1, 2, 3, 5])
+def test_spec_round_trip_any_slice_width(slice_cg):
+    L = make_layer(70, 640, 2, key=(82, slice_cg))
+    img = spec.pack_spec(L.planes, L.g, L.h, slice_cg)
+    planes, g, h = spec.unpack_spec(img)
+    assert np.array_equal(planes, L.planes)
+    # the library unpacker honours the slice width recorded in the header
+    p2, _, _ = rabit.unpack_host(img, 2, 70, 640)
+    assert np.array_equal(p2, L.planes)
+
+
+def test_single_bit_lands_where_the_definition_says():
+    K, M, N = 2, 64, 256
+    planes = make_planes_constant(K, M, N, 0)
+    row, col, k = 37, 203, 1
+    planes[k, row, col // 32] = np.uint32(1 << (col % 32))
+    L = make_layer(M, N, K, key=(83,))
+    img = rabit.pack_host(planes, L.g, L.h)
+    hd = spec.read_header(img)
+    bits = img[hd["off_bits"]:hd["off_g"]]
+    nz = np.flatnonzero(bits)
+    assert nz.size == 1
+    rt, rl = divmod(row, 32); r16, rg = divmod(rl, 2); alo, gq = divmod(r16, 8)
+    cg, cl = divmod(col, 128); cs, rem = divmod(cl, 32); ah, rem = divmod(rem, 16); tq, c = divmod(rem, 4)
+    s, q = divmod(cg, hd["slice_cg"])
+    ncg = min(hd["n_cg"], (s + 1) * hd["slice_cg"]) - s * hd["slice_cg"]
+    tile = K * hd["n_rt"] * s * hd["slice_cg"] + (rt * ncg + q) * K + k
+    off = tile * 512 + 16 * (4 * gq + tq) + 4 * (alo + 2 * ah) + c
+    assert nz[0] == off and bits[off] == 1 << (rg + 2 * cs)
+
+
+def test_scratch_and_padding_are_zero():
+    L = make_layer(40, 160, 2, key=(84,))
+    img = rabit.pack_host(L.planes, L.g, L.h)
+    hd = spec.read_header(img)
+    assert not img[hd["off_partial"]:hd["total_bytes"]].any()
+    g = img[hd["off_g"]:hd["off_h"]].view(np.uint16)[:2 * hd["Mp"]].reshape(2, hd["Mp"])
+    assert not g[:, 40:].any()
+
+
+def test_shape_and_buffer_errors():
+    lib = binding.raw_lib()
+    assert rabit.packed_bytes(2, 64, 48) == 0          # N not a multiple of 32
+    assert rabit.packed_bytes(4, 64, 64) == 0          # K > 3
+    assert rabit.packed_bytes(2, 0, 64) == 0
+    L = make_layer(32, 64, 2, key=(85,))
+    need = rabit.packed_bytes(2, 32, 64)
+    small = np.empty(need - 1, dtype=np.uint8)
+    g16 = L.g.view(np.uint16); h16 = L.h.view(np.uint16)
+    rc = lib.rabit_pack_host(L.planes.ctypes.data, g16.ctypes.data, h16.ctypes.data, 2, 32, 64, small.ctypes.data, small.nbytes)
+    assert rc == -3 and "need" in rabit.last_error()
+    rc = lib.rabit_pack_host(None, g16.ctypes.data, h16.ctypes.data, 2, 32, 64, small.ctypes.data, small.nbytes)
+    assert rc == -1
+    rc = lib.rabit_pack_host(L.planes.ctypes.data, g16.ctypes.data, h16.ctypes.data, 2, 32, 48, small.ctypes.data, small.nbytes)
+    assert rc == -2
+    with pytest.raises(rabit.RabitError):
+        rabit.pack_host(np.zeros((4, 32, 2), np.uint32), np.zeros((4, 32), np.float16), np.zeros((4, 64), np.float16))
+    junk = np.zeros(512, dtype=np.uint8)
+    assert lib.rabit_unpack_host(junk.ctypes.data, junk.nbytes, None, None, None) == -1
+    # host-side argument checks of the device entry points need no GPU
+    assert lib.rabit_linear(None, None, None, 1, None) == -1
+    assert lib.rabit_free(None) == 0
+    assert lib.rabit_layer_K(None) == -1
+    out = ctypes.c_void_p()
+    assert lib.rabit_pack(None, None, None, 2, 32, 64, None, 0, None, ctypes.byref(out)) == -1
+
+
+def test_every_declared_symbol_is_exported():
+    header = open(os.path.join(ROOT, "include", "rabit.h")).read()
+    names = re.findall(r"RABIT_API\s+[\w\s\*]+?\b(rabit_\w+)\s*\(", header)
+    assert len(names) >= 13
+    lib = ctypes.CDLL(rabit.lib_path())
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/rabit.h but not exported"
