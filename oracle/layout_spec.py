@@ -5,7 +5,7 @@ library image can be compared byte for byte.  The paper fixes only the sign -> b
 (Appendix "Weight Packing": +1 -> 0, -1 -> 1); the arrangement below is this build's.
 
 Image = header (256 B) | sign tiles | g fp16 [K][Mp] | h fp16 [K][Np] | fp32 scratch
-[n_slices][Mp] | u32 counters [n_rt]; every section starts on a 256-byte boundary; padding,
+[2][n_slices][Mp] | u32 counters [n_rt]; every section starts on a 256-byte boundary; padding,
 scratch and counters are zero.  Mp = M rounded up to 32, Np = N rounded up to 128; padded
 signs are +1 (bit 0), padded scales 0.
 
@@ -45,7 +45,7 @@ def geometry(K: int, M: int, N: int, slice_cg: int) -> dict:
     geo["off_bits"] = off; off = _align256(off + K * n_rt * n_cg * TILE_BYTES)
     geo["off_g"] = off; off = _align256(off + K * Mp * 2)
     geo["off_h"] = off; off = _align256(off + K * Np * 2)
-    geo["off_partial"] = off; off = _align256(off + n_slices * Mp * 4)
+    geo["off_partial"] = off; off = _align256(off + 2 * n_slices * Mp * 4)
     geo["off_counters"] = off; off = _align256(off + n_rt * 4)
     geo["total_bytes"] = off
     return geo

@@ -19,7 +19,7 @@ struct rabit_layer {
     const uint4* d_bits;         // sign tiles
     const uint16_t* d_g;         // fp16 [K][Mp]
     const uint16_t* d_h;         // fp16 [K][Np]
-    float* d_partial;            // fp32 [n_slices][Mp] reduction scratch (kept zero between calls)
+    float* d_partial;            // fp32 [2][n_slices][Mp] cross-slice partial sums (fully rewritten by every call)
     unsigned int* d_counters;    // u32 [n_rt] arrival counters (kept zero between calls)
 };
 

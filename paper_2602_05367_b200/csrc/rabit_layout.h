@@ -37,6 +37,7 @@
 #define RABIT_HEADER_BYTES 256
 #define RABIT_MAX_K 3
 #define RABIT_MAX_GEMV_BATCH 16
+#define RABIT_PARTIAL_BATCH 2   /* batch rows the cross-slice partial buffer holds */
 
 struct RabitHeader {            // first 256 bytes of a packed image (little endian)
     uint32_t magic;

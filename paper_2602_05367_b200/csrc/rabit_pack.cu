@@ -39,7 +39,7 @@ void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr) {
     hdr->off_bits = off;     off = rabit_align256(off + (size_t)G.K * G.n_rt * G.n_cg * RABIT_TILE_BYTES);
     hdr->off_g = off;        off = rabit_align256(off + (size_t)G.K * G.Mp * 2);
     hdr->off_h = off;        off = rabit_align256(off + (size_t)G.K * G.Np * 2);
-    hdr->off_partial = off;  off = rabit_align256(off + (size_t)G.n_slices * G.Mp * 4);
+    hdr->off_partial = off;  off = rabit_align256(off + (size_t)RABIT_PARTIAL_BATCH * G.n_slices * G.Mp * 4);
     hdr->off_counters = off; off = rabit_align256(off + (size_t)G.n_rt * 4);
     hdr->total_bytes = off;
 }
