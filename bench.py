@@ -1,0 +1,354 @@
+"""Benchmark of the residual-binary linear layer on B200.
+
+Workload (``config.workload``): the seven projections of a Llama-2-7B-shaped decoder layer
+(q,k,v,o 4096->4096; gate,up 4096->11008; down 11008->4096) as K=2 residual-binary layers,
+batch 1, run back to back.  One *step* is one such decoder layer = seven ``rabit_linear``
+calls.  To keep the weights cold in HBM the run rotates over ``--copies`` distinct decoder
+layers (default 32, i.e. the 224 projections of a 7B-shaped stack, 1.6 GB packed, far
+above the 126 MB L2), so every step streams weights that were evicted long ago.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl rabit|reference]
+
+For N > 1 launch under ``torch.distributed.run``; every rank holds its own replica of the
+workload (the path has no exchange step), timing is the max over ranks.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "batch-1 residual-binary GEMV us/layer"
+UNIT = "us/layer"
+WORKLOAD = "llama2-7b decoder layer: 7 residual-binary projections, K=2, batch 1, back to back"
+K_PATHS = 2
+
+
+def layer_bytes(M: int, N: int, batch: int, K: int = K_PATHS) -> int:
+    """Algorithmic bytes of one call: sign bits + fp16 scales + x in + y out."""
+    return K * M * N // 8 + 2 * K * (M + N) + 2 * batch * (M + N)
+
+
+# ---------------------------------------------------------------------------------------
+# clocks sampler (nvidia-smi in the background, as the profiling recipe prescribes)
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int, period_ms: int = 100):
+        self.samples = []   # (t, sm_mhz, max_mhz, {reason: bool})
+        self.proc = None
+        self.thread = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(gpu_index), "-lms", str(period_ms)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm, mx = float(parts[1]), float(parts[2])
+            except ValueError:
+                continue
+            names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+            reasons = {n: parts[5 + i].lower().startswith("active") for i, n in enumerate(names)}
+            self.samples.append((time.time(), sm, mx, reasons))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        reasons = sorted({n for s in inside for n, on in s[3].items() if on})
+        return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": inside[0][2],
+                "reasons": reasons, "samples": len(inside)}
+
+
+# ---------------------------------------------------------------------------------------
+# workload
+# ---------------------------------------------------------------------------------------
+def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: int = 1):
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from synth import llama2_7b_layer_shapes, make_layer, make_x
+
+    shapes = llama2_7b_layer_shapes()
+    layers = []            # [copy][proj] -> RabitLayer
+    for c in range(copies):
+        row = []
+        for p, sh in enumerate(shapes):
+            L = make_layer(sh.M, sh.N, K_PATHS, key=(seed_cfg, c, p))
+            row.append(rabit.rabit_pack(L.planes, L.g, L.h, device=device))
+        layers.append(row)
+    widths = sorted({sh.N for sh in shapes})
+    xs_host = {n: np.stack([make_x(batch, n, key=(seed_cfg, 10_000 + t)) for t in range(tokens)]) for n in widths}
+    xs = {n: torch.from_numpy(a).to(device) for n, a in xs_host.items()}            # [tokens][batch][N]
+    ys = [torch.zeros((batch, sh.M), dtype=torch.float16, device=device) for sh in shapes]
+    return shapes, layers, xs, xs_host, ys
+
+
+def run_step(rabit, shapes, layer_row, xs, ys, token: int):
+    for p, sh in enumerate(shapes):
+        rabit.rabit_linear(layer_row[p], xs[sh.N][token], ys[p])
+
+
+# ---------------------------------------------------------------------------------------
+# the library arm
+# ---------------------------------------------------------------------------------------
+def bench_rabit(args) -> dict:
+    import torch
+    import paper_2602_05367_b200 as rabit
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device(device))
+        dist = dist_mod
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    copies, batch, tokens = args.copies, args.batch, 16
+    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens)
+    step_bytes = sum(layer_bytes(sh.M, sh.N, batch) for sh in shapes)
+    n_proj = len(shapes)
+    stream = torch.cuda.Stream(device)
+
+    # one CUDA graph per decoder-layer copy, and one that walks all copies once
+    def capture(copy_ids):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for c in copy_ids:
+                run_step(rabit, shapes, layers[c], xs, ys, c % tokens)
+        return g
+
+    with torch.cuda.stream(stream):
+        for c in range(copies):                      # also the first-call set-up of every kernel variant
+            run_step(rabit, shapes, layers[c], xs, ys, c % tokens)
+    stream.synchronize()
+    use_graph = not args.no_graph
+    if use_graph:
+        cycle_graph = capture(list(range(copies)))
+        step_graphs = [capture([c]) for c in range(copies)]
+
+    def run_steps(first: int, count: int):
+        """Steps first .. first+count-1; step s uses decoder-layer copy s % copies."""
+        s, end = first, first + count
+        with torch.cuda.stream(stream):
+            while s < end:
+                if not use_graph:
+                    run_step(rabit, shapes, layers[s % copies], xs, ys, (s % copies) % tokens)
+                    s += 1
+                elif s % copies == 0 and end - s >= copies:
+                    cycle_graph.replay(); s += copies
+                else:
+                    step_graphs[s % copies].replay(); s += 1
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    run_steps(0, args.warmup)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+    run_steps(args.warmup, args.steps)
+    with torch.cuda.stream(stream):
+        ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    clocks = sampler.summary(t_wall0, t_wall1) if sampler else None
+    if sampler and clocks["samples"] < 3:
+        # the timed region was shorter than the sampling period: repeat the same work, untimed,
+        # for about a second under the sampler and report the clocks seen there
+        reps = max(1, int(1.0 / max(ms * 1e-3, 1e-4)))
+        t0 = time.time()
+        for _ in range(reps):
+            run_steps(args.warmup, args.steps)
+        torch.cuda.synchronize()
+        clocks = sampler.summary(t0, time.time())
+        clocks["note"] = "sampled over an untimed repeat of the timed region (region shorter than the sampler period)"
+    if sampler:
+        sampler.stop()
+
+    ms_per_step = ms / args.steps
+    us_per_layer = ms_per_step * 1e3 / n_proj
+    gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e = None
+    if rank == 0 or dist is not None:
+        pin_x = {n: torch.from_numpy(a).pin_memory() for n, a in xs_host.items()}
+        pin_y = [torch.empty((batch, sh.M), dtype=torch.float16).pin_memory() for sh in shapes]
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+        def e2e_step(s):
+            c = s % copies
+            with torch.cuda.stream(stream):
+                for p, sh in enumerate(shapes):
+                    rabit.rabit_linear_host(layers[c][p], pin_x[sh.N][c % tokens], pin_y[p], stream=stream.cuda_stream)
+                stream.synchronize()                  # the caller reads y on the host after every step
+        for s in range(min(3 * copies, 100)):
+            e2e_step(s)
+        barrier()
+        t0 = time.perf_counter()
+        with torch.cuda.stream(stream):
+            ev0.record(stream)
+        for s in range(e2e_steps):
+            e2e_step(s)
+        with torch.cuda.stream(stream):
+            ev1.record(stream)
+        barrier()
+        e_ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([e_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": e_ms * 1e3 / e2e_steps / n_proj / world, "unit": UNIT,
+               "h2d_bytes_per_step": int(sum(2 * batch * sh.N for sh in shapes)),
+               "d2h_bytes_per_step": int(sum(2 * batch * sh.M for sh in shapes)),
+               "steps": e2e_steps, "note": "rabit_linear_host per projection: pinned host x -> device, kernel, "
+                                           "y -> pinned host, host synchronises after every step"}
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    result = {
+        "metric": METRIC, "value": us_per_layer / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 tensor-core products of exact fixed-point activations, int32/fp32 accumulate, fp16 in/out",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "copies": copies, "batch": batch, "K": K_PATHS,
+                   "packed_bytes_total": int(step_bytes * copies),
+                   "l2": "inputs larger than L2: rotation over %d distinct decoder layers (%.0f MB)" % (copies, step_bytes * copies / 1e6),
+                   "launch": "CUDA graph replay" if use_graph else "stream launches",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "achieved_hbm_gbs": gbs * world,
+        "tokens_per_s_32_layer_stack": world * 1.0 / (32 * ms_per_step * 1e-3),
+        "gpu_launches": args.steps * n_proj,
+        "clocks": clocks,
+        "e2e": e2e,
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "traffic": None, "peak_source": peak_src,
+                     "note": "algorithmic bytes of the seven layers of a step / device time of a step (launch gaps included)"},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(sample_projections=n_proj)
+    for row in layers:
+        for L in row:
+            L.free()
+    if dist is not None:
+        dist.destroy_process_group()
+    return result if rank == 0 else None
+
+
+# ---------------------------------------------------------------------------------------
+# the oracle, timed as it stands on the host cores
+# ---------------------------------------------------------------------------------------
+def cpu_baseline(sample_projections: int = 7, repeats: int = 1) -> dict:
+    from oracle import rabit_oracle as orc
+    from synth import llama2_7b_layer_shapes, make_layer, make_x
+
+    shapes = llama2_7b_layer_shapes()[:sample_projections]
+    inputs = [(make_layer(sh.M, sh.N, K_PATHS, key=(1, 0, p)), make_x(1, sh.N, key=(1, 10_000))) for p, sh in enumerate(shapes)]
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        for L, x in inputs:
+            orc.linear(L.planes, L.g, L.h, x)
+    dt = (time.perf_counter() - t0) / repeats
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count()
+    return {"value": dt * 1e6 / len(shapes), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "decoder-layer copy 0, its %d projections once each, batch 1 (float64: unpack signs, dense W, product)" % len(shapes)}
+
+
+def bench_reference(args) -> dict:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    per_layer = []
+    base = None
+    for _ in range(max(1, min(args.warmup, 1))):
+        cpu_baseline(sample_projections=1)
+    t0 = time.perf_counter()
+    steps = max(1, min(args.steps, 4))
+    for _ in range(steps):
+        base = cpu_baseline()
+        per_layer.append(base["value"])
+    dt = time.perf_counter() - t0
+    value = float(np.mean(per_layer))
+    base["value"] = value
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / steps, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch": 1, "K": K_PATHS},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32000)
+    ap.add_argument("--warmup", type=int, default=640)
+    ap.add_argument("--impl", default="rabit", choices=["rabit", "reference"])
+    ap.add_argument("--copies", type=int, default=32)
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=2000)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    res = bench_reference(args) if args.impl == "reference" else bench_rabit(args)
+    if res is not None:
+        print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()

@@ -100,6 +100,19 @@ RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16
  */
 RABIT_API int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
+/*
+ * Host-buffer form of rabit_linear (same operation, Section 4.1 forward with the Eq. 2 weight)
+ * for callers whose activations live in host memory:
+ *   x_host  HOST fp16 [batch][N]   (pinned memory makes the copies asynchronous)
+ *   y_host  HOST fp16 [batch][M]
+ *   dev_stage DEVICE, 256-byte aligned, caller-owned, at least rabit_stage_bytes(layer, batch)
+ * Enqueues on `stream`: copy x to the stage, the layer kernel, copy y back.  Returns without
+ * synchronising; y_host is valid once the stream has reached this point.
+ */
+RABIT_API size_t rabit_stage_bytes(const rabit_layer* layer, int batch);
+RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, void* y_host, int batch,
+                      void* dev_stage, size_t dev_stage_bytes, void* stream);
+
 /* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
 RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
                  void* stream);

@@ -25,7 +25,7 @@ class RabitError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(_LIB_PATH):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2602_05367_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python paper_2602_05367_b200/build.py` "
             "(there is no CPU fallback)")
     lib = ctypes.CDLL(_LIB_PATH)
     lib.rabit_layout_version.restype = _c_int
@@ -40,6 +40,10 @@ def _load() -> ctypes.CDLL:
                                _c_void_p, ctypes.POINTER(_c_void_p)]
     lib.rabit_linear.restype = _c_int
     lib.rabit_linear.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
+    lib.rabit_stage_bytes.restype = _c_size_t
+    lib.rabit_stage_bytes.argtypes = [_c_void_p, _c_int]
+    lib.rabit_linear_host.restype = _c_int
+    lib.rabit_linear_host.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]
     lib.rabit_unpack.restype = _c_int
     lib.rabit_unpack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p]
     for name in ("rabit_layer_K", "rabit_layer_M", "rabit_layer_N"):
@@ -50,10 +54,6 @@ def _load() -> ctypes.CDLL:
     lib.rabit_free.restype = _c_int
     lib.rabit_free.argtypes = [_c_void_p]
     lib.rabit_last_error.restype = ctypes.c_char_p
-    if hasattr(lib, "rabit_linear_static_scratch"):
-        lib.rabit_linear_static_scratch.restype = _c_int
-        lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
-        lib.rabit_static_scratch_max_bytes.restype = _c_size_t
     return lib
 
 
@@ -127,6 +127,7 @@ class RabitLayer:
         self._handle = _c_void_p(handle)
         self.dev_buf = dev_buf          # keeps the device memory alive
         self.K, self.M, self.N = K, M, N
+        self._stage = None              # device staging buffer of rabit_linear_host
 
     @property
     def handle(self) -> ctypes.c_void_p:
@@ -149,6 +150,7 @@ class RabitLayer:
             _lib.rabit_free(self._handle)
             self._handle = None
             self.dev_buf = None
+            self._stage = None
 
     def __del__(self):  # pragma: no cover
         try:
@@ -192,6 +194,28 @@ def rabit_linear(layer: RabitLayer, x, y=None, stream: Optional[int] = None):
     st = torch.cuda.current_stream(x.device).cuda_stream if stream is None else stream
     _check(_lib.rabit_linear(layer.handle, _c_void_p(xb.data_ptr()), _c_void_p(y.data_ptr()), batch, _c_void_p(st)))
     return y if x.dim() == 2 else y.view(-1)
+
+
+def rabit_linear_host(layer: RabitLayer, x_host, y_host, stream: Optional[int] = None):
+    """Host-buffer form: x_host / y_host are CPU float16 tensors (pinned for asynchronous copies)
+    of shape [batch][N] (or [N]) and [batch][M]; the copies and the kernel are enqueued on the
+    stream and the call returns without synchronising."""
+    import torch
+
+    if x_host.dtype != torch.float16 or x_host.is_cuda or not x_host.is_contiguous():
+        raise ValueError("x_host must be a contiguous CPU float16 tensor")
+    if y_host.dtype != torch.float16 or y_host.is_cuda or not y_host.is_contiguous():
+        raise ValueError("y_host must be a contiguous CPU float16 tensor")
+    batch = 1 if x_host.dim() == 1 else x_host.shape[0]
+    if x_host.numel() != batch * layer.N or y_host.numel() != batch * layer.M:
+        raise ValueError("x_host / y_host sizes do not match the layer")
+    need = int(_lib.rabit_stage_bytes(layer.handle, batch))
+    if layer._stage is None or layer._stage.numel() < need:
+        layer._stage = torch.empty(need, dtype=torch.uint8, device=layer.dev_buf.device)
+    st = torch.cuda.current_stream(layer.dev_buf.device).cuda_stream if stream is None else stream
+    _check(_lib.rabit_linear_host(layer.handle, _c_void_p(x_host.data_ptr()), _c_void_p(y_host.data_ptr()), batch,
+                                  _c_void_p(layer._stage.data_ptr()), need, _c_void_p(st)))
+    return y_host
 
 
 def rabit_free(layer: RabitLayer) -> None:

@@ -1,6 +1,7 @@
 """Builds librabit.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-Usage: ``python -m paper_2602_05367_b200.build [--force] [--verbose]``.
+Usage: ``python paper_2602_05367_b200/build.py [--force] [--verbose]`` (run as a script: importing the
+package needs the library to exist already).
 """
 from __future__ import annotations
 
@@ -11,8 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librabit.so")
-SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemm_tc.cu",
-           "rabit_noalloc.cu"]
+SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemm_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-shared", "-cudart", "static",

@@ -115,6 +115,32 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
     return RABIT_OK;
 }
 
+extern "C" size_t rabit_stage_bytes(const rabit_layer* layer, int batch) {
+    if (!layer || batch < 1) return 0;
+    return rabit_align256((size_t)batch * layer->geom.N * 2) + rabit_align256((size_t)batch * layer->geom.M * 2);
+}
+
+extern "C" int rabit_linear_host(const rabit_layer* layer, const void* x_host, void* y_host, int batch,
+                                 void* dev_stage, size_t dev_stage_bytes, void* stream) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_host: layer is NULL");
+    if (!x_host || !y_host || !dev_stage) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_host: null pointer");
+    if (batch < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_host: batch must be >= 1 (got %d)", batch);
+    if (((uintptr_t)dev_stage & 255u) != 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_host: dev_stage must be 256-byte aligned");
+    const size_t need = rabit_stage_bytes(layer, batch);
+    if (dev_stage_bytes < need)
+        return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_linear_host: stage holds %zu bytes, need %zu", dev_stage_bytes, need);
+    const size_t xb = (size_t)batch * layer->geom.N * 2, yb = (size_t)batch * layer->geom.M * 2;
+    char* dx = (char*)dev_stage;
+    char* dy = dx + rabit_align256(xb);
+    cudaStream_t st = (cudaStream_t)stream;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(dx, x_host, xb, cudaMemcpyHostToDevice, st));
+    int rc = rabit_linear(layer, dx, dy, batch, stream);
+    if (rc != RABIT_OK) return rc;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(y_host, dy, yb, cudaMemcpyDeviceToHost, st));
+    return RABIT_OK;
+}
+
 extern "C" int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out, void* stream) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack: layer is NULL");

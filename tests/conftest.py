@@ -8,6 +8,21 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _ensure_library():
+    """Build librabit.so in-tree when it is missing or older than its sources (the built
+    file is not kept in the history).  The build script is loaded by path because importing
+    the package needs the library to exist."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location(
+        "_rabit_build", os.path.join(ROOT, "paper_2602_05367_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build(force=False)
+
+
+_ensure_library()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 

@@ -145,3 +145,19 @@ def test_argument_errors_on_device():
                         2, 64, 128, vp(p), 16, None, ctypes.byref(out))
     assert rc == -3                                                                     # device buffer too small
     layer.free()
+
+
+@pytest.mark.parametrize("batch", [1, 3])
+def test_host_buffer_entry_point(batch):
+    """rabit_linear_host: pinned host x in, pinned host y out, copies enqueued by the library."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(200, 640, 2, key=(78,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    xn = make_x(batch, 640, key=(78, batch))
+    xh = torch.from_numpy(xn).pin_memory()
+    yh = torch.zeros((batch, 200), dtype=torch.float16).pin_memory()
+    rabit.rabit_linear_host(layer, xh, yh)
+    torch.cuda.synchronize()
+    check_against_oracle(L, xn, yh.numpy())
+    layer.free()
