@@ -55,7 +55,12 @@ extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint1
 
     rabit_layer* L = new (std::nothrow) rabit_layer;
     if (!L) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: out of host memory");
-    L->geom = G;
+    RabitHeader packed_hdr;
+    std::memcpy(&packed_hdr, image.data(), sizeof(packed_hdr));
+    if (!rabit_geom_from_header(packed_hdr, &L->geom)) {
+        delete L;
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: internal error, packed header unreadable");
+    }
     L->device = attr.device;
     L->variant = 0;
     L->sm_count = 0;
@@ -67,6 +72,7 @@ extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint1
     L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
     L->d_partial = (float*)(L->dev_base + hdr.off_partial);
     L->d_counters = (unsigned int*)(L->dev_base + hdr.off_counters);
+    L->d_status = L->d_counters + G.n_rt;
     *out = L;
     return RABIT_OK;
 }
@@ -100,7 +106,10 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
         case 2:
             if (!rabit_gemv_mma_supports(*layer, batch))
                 return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: integer-MMA GEMV cannot run batch %d", batch);
-            e = rabit_launch_gemv_mma(*layer, x, y, batch, st);
+            e = cudaSuccess;
+            for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += 2)      // two batch rows share one pass over the weights
+                e = rabit_launch_gemv_mma(*layer, (const char*)x + (size_t)b0 * G.N * 2, (char*)y + (size_t)b0 * G.M * 2,
+                                          batch - b0 >= 2 ? 2 : 1, st);
             break;
         case 3:
             if (!rabit_gemm_tc_supports(*layer, batch))

@@ -18,9 +18,10 @@ struct rabit_layer {
     size_t dev_bytes;
     const uint4* d_bits;         // sign tiles
     const uint16_t* d_g;         // fp16 [K][Mp]
-    const uint16_t* d_h;         // fp16 [K][Np]
-    float* d_partial;            // fp32 [2][n_slices][Mp] cross-slice partial sums (fully rewritten by every call)
-    unsigned int* d_counters;    // u32 [n_rt] arrival counters (kept zero between calls)
+    const uint16_t* d_h;         // fp16 [K][N]
+    float* d_partial;            // fp32 [n_rt*K + RABIT_MAX_GRID][RABIT_PARTIAL_BATCH][128] cross-CTA partial sums
+    unsigned int* d_counters;    // u32 [n_rt] arrival counters (kept zero between calls), then one status word
+    unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
 };
 
 // error reporting (thread-local message); returns `code`
@@ -34,8 +35,9 @@ void rabit_clear_error();
     } while (0)
 
 // geometry / layout (rabit_pack.cu)
-bool rabit_make_geom(int K, int M, int N, RabitGeom* out);
+bool rabit_make_geom(int K, int M, int N, RabitGeom* out);          // hmax left at 0
 void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr);
+bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out); // validates magic, version and shape
 
 // kernel launchers; each enqueues on `stream` and returns a cudaError_t from the launch
 cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);

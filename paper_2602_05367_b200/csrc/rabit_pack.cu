@@ -2,16 +2,29 @@
 // (step "pack" of the layer; Appendix "Weight Packing" of the paper fixes only the
 // sign -> bit rule, the tile arrangement is described in rabit_layout.h).
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <thread>
 #include <vector>
 
 #include "rabit_internal.h"
 
-static int choose_slice_cg(int /*K*/, int /*M*/, int N_cg) {
-    // Column groups (of 128 inputs) per slice.  A slice is the unit for which a CTA prepares
-    // the fixed-point activations once; 4 groups = 512 inputs.
-    return std::min(N_cg, 4);
+static float half_bits_to_float(uint16_t v) {
+    const uint32_t sign = (uint32_t)(v & 0x8000u) << 16;
+    const int e = (v >> 10) & 0x1F;
+    uint32_t m = v & 0x3FFu, bits;
+    if (e == 0) {
+        if (m == 0) bits = sign;
+        else {                                  // subnormal: normalise
+            int sh = 0;
+            while (!(m & 0x400u)) { m <<= 1; ++sh; }
+            bits = sign | ((uint32_t)(127 - 15 - sh + 1) << 23) | ((m & 0x3FFu) << 13);
+        }
+    } else if (e == 31) bits = sign | 0x7F800000u | (m << 13);
+    else bits = sign | ((uint32_t)(e - 15 + 127) << 23) | (m << 13);
+    float f;
+    std::memcpy(&f, &bits, 4);
+    return f;
 }
 
 bool rabit_make_geom(int K, int M, int N, RabitGeom* out) {
@@ -20,11 +33,9 @@ bool rabit_make_geom(int K, int M, int N, RabitGeom* out) {
     RabitGeom G;
     G.K = K; G.M = M; G.N = N;
     G.Mp = (M + RABIT_TILE_ROWS - 1) / RABIT_TILE_ROWS * RABIT_TILE_ROWS;
-    G.Np = (N + RABIT_TILE_COLS - 1) / RABIT_TILE_COLS * RABIT_TILE_COLS;
     G.n_rt = G.Mp / RABIT_TILE_ROWS;
-    G.n_cg = G.Np / RABIT_TILE_COLS;
-    G.slice_cg = choose_slice_cg(K, M, G.n_cg);
-    G.n_slices = (G.n_cg + G.slice_cg - 1) / G.slice_cg;
+    G.n_ct = N / RABIT_TILE_COLS;
+    for (int k = 0; k < RABIT_MAX_K; ++k) G.hmax[k] = 0.f;
     *out = G;
     return true;
 }
@@ -33,15 +44,26 @@ void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr) {
     std::memset(hdr, 0, sizeof(RabitHeader));
     hdr->magic = RABIT_MAGIC;
     hdr->version = RABIT_LAYOUT_VERSION;
-    hdr->K = G.K; hdr->M = G.M; hdr->N = G.N; hdr->Mp = G.Mp; hdr->Np = G.Np;
-    hdr->n_rt = G.n_rt; hdr->n_cg = G.n_cg; hdr->slice_cg = G.slice_cg; hdr->n_slices = G.n_slices;
+    hdr->K = G.K; hdr->M = G.M; hdr->N = G.N; hdr->Mp = G.Mp;
+    hdr->n_rt = G.n_rt; hdr->n_ct = G.n_ct;
+    hdr->max_grid = RABIT_MAX_GRID;
+    hdr->partial_batch = RABIT_PARTIAL_BATCH;
+    for (int k = 0; k < G.K; ++k) std::memcpy(&hdr->hmax_bits[k], &G.hmax[k], 4);
     size_t off = RABIT_HEADER_BYTES;
-    hdr->off_bits = off;     off = rabit_align256(off + (size_t)G.K * G.n_rt * G.n_cg * RABIT_TILE_BYTES);
+    hdr->off_bits = off;     off = rabit_align256(off + (size_t)G.K * G.n_rt * G.n_ct * RABIT_TILE_BYTES);
     hdr->off_g = off;        off = rabit_align256(off + (size_t)G.K * G.Mp * 2);
-    hdr->off_h = off;        off = rabit_align256(off + (size_t)G.K * G.Np * 2);
-    hdr->off_partial = off;  off = rabit_align256(off + (size_t)RABIT_PARTIAL_BATCH * G.n_slices * G.Mp * 4);
-    hdr->off_counters = off; off = rabit_align256(off + (size_t)G.n_rt * 4);
+    hdr->off_h = off;        off = rabit_align256(off + (size_t)G.K * G.N * 2);
+    hdr->off_partial = off;  off = rabit_align256(off + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID) * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS * 4);
+    hdr->off_counters = off; off = rabit_align256(off + (size_t)G.n_rt * 4 + 4);   // + one status word
     hdr->total_bytes = off;
+}
+
+bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out) {
+    if (hdr.magic != RABIT_MAGIC || hdr.version != RABIT_LAYOUT_VERSION) return false;
+    if (!rabit_make_geom((int)hdr.K, (int)hdr.M, (int)hdr.N, out)) return false;
+    if (hdr.max_grid != RABIT_MAX_GRID || hdr.partial_batch != RABIT_PARTIAL_BATCH) return false;
+    for (int k = 0; k < out->K; ++k) std::memcpy(&out->hmax[k], &hdr.hmax_bits[k], 4);
+    return true;
 }
 
 extern "C" int rabit_layout_version(void) { return RABIT_LAYOUT_VERSION; }
@@ -60,24 +82,23 @@ static inline uint64_t spread8(uint32_t v) {
     return ((m + 0x7F7F7F7F7F7F7F7FULL) >> 7) & 0x0101010101010101ULL;
 }
 
-static void pack_tile(const RabitGeom& G, const uint32_t* plane /*[M][N/32]*/, int rt, int cg, uint8_t* dst) {
+static void pack_tile(const RabitGeom& G, const uint32_t* plane /*[M][N/32]*/, int rt, int ct, uint8_t* dst) {
     const int words_per_row = G.N / 32;
-    for (int r16 = 0; r16 < 16; ++r16) {
-        // bytes[b] collects, for source bit position b, the 8 bits (p = row parity + 2 * column set)
+    for (int r16 = 0; r16 < 16; ++r16) {            // r16 = gq + 8 * (a & 1): row inside a 16-row block
+        // bytes[q] byte b collects, for column 8q + b of the tile, bit p <- row 16p + r16
         uint64_t bytes[4] = {0, 0, 0, 0};
         for (int p = 0; p < 8; ++p) {
-            int row = rt * RABIT_TILE_ROWS + 2 * r16 + (p & 1);
-            int word = cg * 4 + (p >> 1);
+            const int row = rt * RABIT_TILE_ROWS + 16 * p + r16;
             uint32_t s = 0;
-            if (row < G.M && word < words_per_row) s = plane[(size_t)row * words_per_row + word];
+            if (row < G.M) s = plane[(size_t)row * words_per_row + ct];
             for (int q = 0; q < 4; ++q) bytes[q] |= spread8(s >> (8 * q)) << p;
         }
         const int gq = r16 & 7, alo = r16 >> 3;
-        for (int b4 = 0; b4 < 8; ++b4) {            // 4 consecutive source bit positions = one tq
-            int b = b4 * 4;
-            int ah = b >> 4, tq = (b >> 2) & 3;
-            int a = alo | (ah << 1);
-            uint32_t v = (uint32_t)(bytes[b >> 3] >> (8 * (b & 7)));
+        for (int j4 = 0; j4 < 8; ++j4) {            // 4 consecutive columns = the four bytes of one word
+            const int j = j4 * 4;
+            const int ah = j >> 4, tq = (j >> 2) & 3;
+            const int a = alo | (ah << 1);
+            const uint32_t v = (uint32_t)(bytes[j >> 3] >> (8 * (j & 7)));
             std::memcpy(dst + (4 * gq + tq) * 16 + a * 4, &v, 4);
         }
     }
@@ -90,6 +111,14 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
     RabitGeom G;
     if (!rabit_make_geom(K, M, N, &G))
         return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_pack_host: unsupported shape K=%d M=%d N=%d (need 1<=K<=3, M>=1, N%%32==0)", K, M, N);
+    for (int k = 0; k < K; ++k) {
+        float m = 0.f;
+        for (int j = 0; j < N; ++j) {
+            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
+            if (m == m && (v > m || v != v)) m = v;   // a NaN scale makes the bound NaN
+        }
+        G.hmax[k] = m;
+    }
     RabitHeader hdr;
     rabit_fill_header(G, &hdr);
     if (out_bytes < hdr.total_bytes)
@@ -101,18 +130,13 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
     uint8_t* bits = base + hdr.off_bits;
     const size_t plane_words = (size_t)M * (N / 32);
     int nthreads = (int)std::min<unsigned>(std::max(1u, std::thread::hardware_concurrency()), 32u);
-    if ((size_t)G.n_rt * G.n_cg < 4096) nthreads = 1;
+    if ((size_t)G.n_rt * G.n_ct < 4096) nthreads = 1;
     auto work = [&](int tid) {
         for (int rt = tid; rt < G.n_rt; rt += nthreads)
-            for (int s = 0; s < G.n_slices; ++s) {
-                int ncg = rabit_slice_ncg(G, s);
-                for (int q = 0; q < ncg; ++q)
-                    for (int k = 0; k < K; ++k) {
-                        size_t ti = rabit_tile_index(G, s, rt, q, k);
-                        pack_tile(G, planes + (size_t)k * plane_words, rt, s * G.slice_cg + q,
-                                  bits + ti * RABIT_TILE_BYTES);
-                    }
-            }
+            for (int k = 0; k < K; ++k)
+                for (int ct = 0; ct < G.n_ct; ++ct)
+                    pack_tile(G, planes + (size_t)k * plane_words, rt, ct,
+                              bits + rabit_tile_pos(G, rt, k, ct) * RABIT_TILE_BYTES);
     };
     if (nthreads == 1) {
         work(0);
@@ -125,7 +149,7 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
     uint16_t* hp = (uint16_t*)(base + hdr.off_h);
     for (int k = 0; k < K; ++k) {
         std::memcpy(gp + (size_t)k * G.Mp, g + (size_t)k * M, (size_t)M * 2);
-        std::memcpy(hp + (size_t)k * G.Np, h + (size_t)k * N, (size_t)N * 2);
+        std::memcpy(hp + (size_t)k * N, h + (size_t)k * N, (size_t)N * 2);
     }
     return RABIT_OK;
 }
@@ -137,49 +161,40 @@ extern "C" int rabit_unpack_host(const void* image, size_t image_bytes,
     if (image_bytes < sizeof(RabitHeader)) return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_unpack_host: image smaller than its header");
     RabitHeader hdr;
     std::memcpy(&hdr, image, sizeof(hdr));
-    if (hdr.magic != RABIT_MAGIC || hdr.version != RABIT_LAYOUT_VERSION)
-        return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack_host: not a packed image of layout version %d", RABIT_LAYOUT_VERSION);
     RabitGeom G;
-    if (!rabit_make_geom((int)hdr.K, (int)hdr.M, (int)hdr.N, &G))
-        return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack_host: header holds an unsupported shape");
-    G.slice_cg = (int)hdr.slice_cg;
-    if (G.slice_cg < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack_host: bad slice width in header");
-    G.n_slices = (G.n_cg + G.slice_cg - 1) / G.slice_cg;
+    if (!rabit_geom_from_header(hdr, &G))
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack_host: not a packed image of layout version %d", RABIT_LAYOUT_VERSION);
     if (image_bytes < hdr.total_bytes) return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_unpack_host: image truncated");
     const uint8_t* base = (const uint8_t*)image;
     const int K = G.K, M = G.M, N = G.N, words_per_row = N / 32;
     if (planes_out) {
         std::memset(planes_out, 0, (size_t)K * M * words_per_row * 4);
         const uint8_t* bits = base + hdr.off_bits;
-        for (int s = 0; s < G.n_slices; ++s) {
-            int ncg = rabit_slice_ncg(G, s);
-            for (int rt = 0; rt < G.n_rt; ++rt)
-                for (int q = 0; q < ncg; ++q)
-                    for (int k = 0; k < K; ++k) {
-                        const uint8_t* tile = bits + rabit_tile_index(G, s, rt, q, k) * RABIT_TILE_BYTES;
-                        int cg = s * G.slice_cg + q;
-                        for (int lane = 0; lane < 32; ++lane)
-                            for (int a = 0; a < 4; ++a)
-                                for (int c = 0; c < 4; ++c) {
-                                    uint8_t byte = tile[lane * 16 + a * 4 + c];
-                                    if (!byte) continue;
-                                    int gq = lane >> 2, tq = lane & 3;
-                                    for (int p = 0; p < 8; ++p) {
-                                        if (!((byte >> p) & 1)) continue;
-                                        int row = rt * 32 + 2 * (gq + 8 * (a & 1)) + (p & 1);
-                                        int col = cg * 128 + 32 * (p >> 1) + 16 * (a >> 1) + 4 * tq + c;
-                                        if (row < M && col < N)
-                                            planes_out[((size_t)k * M + row) * words_per_row + col / 32] |= 1u << (col % 32);
-                                    }
+        for (int rt = 0; rt < G.n_rt; ++rt)
+            for (int k = 0; k < K; ++k)
+                for (int ct = 0; ct < G.n_ct; ++ct) {
+                    const uint8_t* tile = bits + rabit_tile_pos(G, rt, k, ct) * RABIT_TILE_BYTES;
+                    for (int lane = 0; lane < 32; ++lane)
+                        for (int a = 0; a < 4; ++a)
+                            for (int c = 0; c < 4; ++c) {
+                                const uint8_t byte = tile[lane * 16 + a * 4 + c];
+                                if (!byte) continue;
+                                const int gq = lane >> 2, tq = lane & 3;
+                                for (int p = 0; p < 8; ++p) {
+                                    if (!((byte >> p) & 1)) continue;
+                                    const int row = rt * RABIT_TILE_ROWS + 16 * p + gq + 8 * (a & 1);
+                                    const int col = ct * RABIT_TILE_COLS + 16 * (a >> 1) + 4 * tq + c;
+                                    if (row < M)
+                                        planes_out[((size_t)k * M + row) * words_per_row + col / 32] |= 1u << (col % 32);
                                 }
-                    }
-        }
+                            }
+                }
     }
     const uint16_t* gp = (const uint16_t*)(base + hdr.off_g);
     const uint16_t* hp = (const uint16_t*)(base + hdr.off_h);
     for (int k = 0; k < K; ++k) {
         if (g_out) std::memcpy(g_out + (size_t)k * M, gp + (size_t)k * G.Mp, (size_t)M * 2);
-        if (h_out) std::memcpy(h_out + (size_t)k * N, hp + (size_t)k * G.Np, (size_t)N * 2);
+        if (h_out) std::memcpy(h_out + (size_t)k * N, hp + (size_t)k * N, (size_t)N * 2);
     }
     return RABIT_OK;
 }

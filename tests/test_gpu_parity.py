@@ -16,6 +16,7 @@ VARIANTS = [0, 1, 2]   # automatic, plain sign-select, integer-MMA GEMV
 
 SMALL = [  # several tiles plus ragged tails in both dimensions
     (2, 32, 128), (2, 100, 160), (2, 256, 1184), (3, 96, 640), (1, 33, 96), (2, 160, 2080), (2, 1000, 512),
+    (1, 128, 32), (2, 129, 32), (3, 700, 8192), (2, 2500, 96),
 ]
 
 

@@ -25,7 +25,7 @@ def test_library_image_equals_spec(K, M, N):
     img = rabit.pack_host(L.planes, L.g, L.h)
     hd = spec.read_header(img)
     assert hd["magic"] == spec.MAGIC and hd["version"] == rabit.layout_version() == spec.VERSION
-    want = spec.pack_spec(L.planes, L.g, L.h, hd["slice_cg"])
+    want = spec.pack_spec(L.planes, L.g, L.h)
     assert img.nbytes == want.nbytes == rabit.packed_bytes(K, M, N)
     assert np.array_equal(img, want)
 
@@ -45,21 +45,31 @@ def test_round_trip_bit_exact(K, M, N):
         assert np.array_equal(h2.view(np.uint16), L.h.view(np.uint16))
 
 
-@pytest.mark.parametrize("slice_cg", [1, 2, 3, 5])
-def test_spec_round_trip_any_slice_width(slice_cg):
-    L = make_layer(70, 640, 2, key=(82, slice_cg))
-    img = spec.pack_spec(L.planes, L.g, L.h, slice_cg)
+def test_spec_round_trip_and_library_reads_spec_image():
+    L = make_layer(70, 640, 2, key=(82,))
+    img = spec.pack_spec(L.planes, L.g, L.h)
     planes, g, h = spec.unpack_spec(img)
     assert np.array_equal(planes, L.planes)
-    # the library unpacker honours the slice width recorded in the header
+    assert np.array_equal(g.view(np.uint16), L.g.view(np.uint16)) and np.array_equal(h.view(np.uint16), L.h.view(np.uint16))
     p2, _, _ = rabit.unpack_host(img, 2, 70, 640)
     assert np.array_equal(p2, L.planes)
 
 
+def test_header_records_largest_input_scale():
+    L = make_layer(40, 96, 3, key=(86,))
+    L.h[1, 17] = np.float16(-7.5)          # the bound uses |h|
+    L.h[2, :] = np.float16(0.0)
+    L.h[2, 5] = np.float16(6e-8)           # a subnormal fp16
+    hd = spec.read_header(rabit.pack_host(L.planes, L.g, L.h))
+    got = np.array([hd["hmax0"], hd["hmax1"], hd["hmax2"]], dtype=np.uint32).view(np.float32)
+    want = np.abs(L.h.astype(np.float32)).max(axis=1)
+    assert np.array_equal(got, want) and got[1] == 7.5 and hd["hmax3"] == 0
+
+
 def test_single_bit_lands_where_the_definition_says():
-    K, M, N = 2, 64, 256
+    K, M, N = 2, 200, 256
     planes = make_planes_constant(K, M, N, 0)
-    row, col, k = 37, 203, 1
+    row, col, k = 45, 203, 1
     planes[k, row, col // 32] = np.uint32(1 << (col % 32))
     L = make_layer(M, N, K, key=(83,))
     img = rabit.pack_host(planes, L.g, L.h)
@@ -67,13 +77,11 @@ def test_single_bit_lands_where_the_definition_says():
     bits = img[hd["off_bits"]:hd["off_g"]]
     nz = np.flatnonzero(bits)
     assert nz.size == 1
-    rt, rl = divmod(row, 32); r16, rg = divmod(rl, 2); alo, gq = divmod(r16, 8)
-    cg, cl = divmod(col, 128); cs, rem = divmod(cl, 32); ah, rem = divmod(rem, 16); tq, c = divmod(rem, 4)
-    s, q = divmod(cg, hd["slice_cg"])
-    ncg = min(hd["n_cg"], (s + 1) * hd["slice_cg"]) - s * hd["slice_cg"]
-    tile = K * hd["n_rt"] * s * hd["slice_cg"] + (rt * ncg + q) * K + k
+    rt, rl = divmod(row, 128); p, r16 = divmod(rl, 16); alo, gq = divmod(r16, 8)
+    ct, cl = divmod(col, 32); ah, rem = divmod(cl, 16); tq, c = divmod(rem, 4)
+    tile = (rt * K + k) * hd["n_ct"] + ct
     off = tile * 512 + 16 * (4 * gq + tq) + 4 * (alo + 2 * ah) + c
-    assert nz[0] == off and bits[off] == 1 << (rg + 2 * cs)
+    assert nz[0] == off and bits[off] == 1 << p
 
 
 def test_scratch_and_padding_are_zero():
