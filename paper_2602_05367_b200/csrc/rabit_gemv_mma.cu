@@ -15,14 +15,14 @@
 // 1/sigma, g_k and the path sum in fp32.  The roundings are T (at most 2^-31 of the bound
 // per term), the fp32 epilogue and the final fp16 store.
 //
-// Structure of a CTA (12 warps):
+// Structure of a CTA (10 warps, two CTAs per SM):
 //   * The tiles of the layer are numbered in layout order; CTA c owns positions
 //     [c*T/G, (c+1)*T/G), one contiguous byte range, so the split is even for every shape.
 //   * One elected thread streams that range with bulk asynchronous copies into a ring of
 //     8 KB stages (mbarrier transaction counts).  The copies for the first ring-full are
 //     issued BEFORE the programmatic-dependency wait: weights never depend on the previous
 //     kernel in the stream, so they stream in while that kernel is still finishing.
-//   * Four builder warps turn x and h into the digit table of each stage (the B fragments,
+//   * Two builder warps turn x and h into the digit table of each stage (the B fragments,
 //     in fragment order) plus the per-tile sum of T, one stage ahead of the consumers.
 //   * Eight MMA warps take the tiles of a stage round-robin: one 128-bit shared-memory read
 //     of weights, one 64-bit read of digits, 32 ANDs and 8 MMAs per 4096 weights.
@@ -39,12 +39,29 @@
 namespace {
 
 constexpr int kMmaWarps = 8;
-constexpr int kBuildWarps = 4;
+constexpr int kBuildWarps = 2;
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kThreads = (kMmaWarps + kBuildWarps) * 32;
 constexpr int kStageTiles = 16;
 constexpr int kRing = 8;
+constexpr int kBuildAhead = 3;                          // stages of raw x / h a builder lane keeps in flight
 constexpr long long kWaitLimitCycles = 1LL << 31;       // about one second
+
+// Division of a 31-bit dividend by a constant known at launch: n / d = (umulhi(n, mul) + n) >> shr.
+struct FastDiv {
+    unsigned int mul, shr, d;
+};
+__host__ inline FastDiv make_fastdiv(unsigned int d) {
+    FastDiv f;
+    f.d = d;
+    unsigned int l = 0;
+    while ((1ull << l) < d) ++l;                      // ceil(log2 d)
+    f.shr = l;
+    f.mul = (unsigned int)((((1ull << l) - d) << 32) / d + 1);
+    return f;
+}
+__device__ __forceinline__ int fdiv(int n, const FastDiv& f) { return (int)((__umulhi((unsigned int)n, f.mul) + (unsigned int)n) >> f.shr); }
+__device__ __forceinline__ int fmod(int n, const FastDiv& f) { return n - fdiv(n, f) * (int)f.d; }
 
 struct GemvParams {
     RabitGeom G;
@@ -56,20 +73,22 @@ struct GemvParams {
     float* partial;          // [n_rt*K + grid][RABIT_PARTIAL_BATCH][128]
     unsigned int* counters;  // [n_rt]
     unsigned int* status;
-    long long n_tiles;       // n_rt * K * n_ct
+    int n_tiles;             // n_rt * K * n_ct (< 2^31)
+    int q, r;                // n_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
+    FastDiv div_c, div_k, div_q, div_q1;   // by n_ct, K, q, q + 1
 };
 
 template <int NB>
 struct __align__(128) Smem {
     uint4 bits[kRing][kStageTiles][32];
     uint2 table[kRing][kStageTiles][NB * 16];           // word pair of lane l (n = l >> 2, tq = l & 3) at index l
-    long long sum_t[kRing][kStageTiles][NB];
+    int sum_t[kRing][kStageTiles][NB][4];               // sum of T over columns 8v .. 8v+7 of the tile, v = 0..3
     float red[kMmaWarps][NB][RABIT_TILE_ROWS];
     unsigned long long full[kRing];
     unsigned long long empty[kRing];
     unsigned int xmax_bits[NB];
     int abort_flag;
-    int is_last;
+    int flag[kMmaThreads];                              // per segment: did this CTA complete the row tile
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -108,10 +127,14 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// CTA that owns tile position p when T tiles are split over G CTAs as [c*T/G, (c+1)*T/G).
-__device__ __forceinline__ int cta_of(long long p, long long T, int G) { return (int)(((p + 1) * G - 1) / T); }
+// Even split of the tile positions: CTA c owns [c*q + min(c, r), (c+1)*q + min(c+1, r)).
+__device__ __forceinline__ int range_lo(int c, int q, int r) { return c * q + min(c, r); }
+__device__ __forceinline__ int cta_of(int p, const GemvParams& P) {
+    const int big = P.r * (P.q + 1);             // positions owned by the CTAs that have q+1 tiles
+    return p < big ? fdiv(p, P.div_q1) : P.r + fdiv(p - big, P.div_q);
+}
 
-// sigma = 2^s with |h x| * sigma < 2^30 for every column; inv = 2^-s (NaN if the inputs are not finite).
+// sigma = 2^s with |h x| * sigma < 2^28 for every column; inv = 2^-s (NaN if the inputs are not finite).
 __device__ __forceinline__ void choose_scale(unsigned int xmax_bits, float hmax, float& sigma, float& inv) {
     const float xm = __half2float(__ushort_as_half((unsigned short)xmax_bits));
     const float bound = xm * hmax;
@@ -121,7 +144,7 @@ __device__ __forceinline__ void choose_scale(unsigned int xmax_bits, float hmax,
     }
     if (bound == 0.f) { sigma = 1.f; inv = 1.f; return; }
     const int e = (__float_as_int(bound) >> 23) & 0xFF;                         // bound < 2^(e - 126)
-    int s = 156 - e;                                                            // 30 - (e - 126)
+    int s = 154 - e;                                                            // 28 - (e - 126)
     s = s > 120 ? 120 : s;
     sigma = __int_as_float((s + 127) << 23);
     inv = __int_as_float((127 - s) << 23);
@@ -135,11 +158,8 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     const RabitGeom& G = P.G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int C = G.n_ct;
-    const long long T = P.n_tiles;
-    const int grid = gridDim.x;
-    const long long lo = (long long)blockIdx.x * T / grid;
-    const long long hi = (long long)(blockIdx.x + 1) * T / grid;
-    const int n_tiles = (int)(hi - lo);
+    const int lo = range_lo(blockIdx.x, P.q, P.r);
+    const int n_tiles = range_lo(blockIdx.x + 1, P.q, P.r) - lo;
     const int n_stages = (n_tiles + kStageTiles - 1) / kStageTiles;
     volatile int* abort_flag = &S.abort_flag;
 
@@ -151,22 +171,54 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         }
         for (int b = 0; b < NB; ++b) S.xmax_bits[b] = 0;
         S.abort_flag = 0;
-        S.is_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    // ---- weights of the first ring-full start streaming before anything that depends on the stream's past
-    const int prefetched = n_stages < kRing ? n_stages : kRing;
+    // ---- everything that does not depend on the stream's past starts now: the first ring-full of
+    //      weights, the first input scales of the builder lanes, the first output scales
     if (tid == kMmaThreads) {
+        const int prefetched = n_stages < kRing ? n_stages : kRing;
         for (int i = 0; i < prefetched; ++i) {
             const int tiles = min(kStageTiles, n_tiles - i * kStageTiles);
             const uint32_t bar = smem_u32(&S.full[i]);
             mbar_expect_tx(bar, tiles * RABIT_TILE_BYTES);
-            bulk_g2s(smem_u32(&S.bits[i][0][0]), P.bits + (lo + (long long)i * kStageTiles) * RABIT_TILE_BYTES,
+            bulk_g2s(smem_u32(&S.bits[i][0][0]), P.bits + ((size_t)lo + (size_t)i * kStageTiles) * RABIT_TILE_BYTES,
                      tiles * RABIT_TILE_BYTES, bar);
         }
     }
+    // Builder lanes: lane index bi = 0..63 of the two builder warps takes tile bi >> 2 of every stage
+    // and columns 8*(bi & 3) .. +7 of it.
+    const int bw = warp - kMmaWarps;
+    const int bi = ((bw & 1) << 5) | lane;
+    const int bj = bi >> 2, bv = bi & 3;
+    int pf_ct = 0, pf_k = 0, pf_stage = 0;           // (column tile, path, stage) of the next prefetch
+    uint4 hq[kBuildAhead];
+    if (warp >= kMmaWarps) {
+        const int p0 = lo + bj;
+        pf_ct = fmod(p0, P.div_c);
+        pf_k = fmod(fdiv(p0, P.div_c), P.div_k);
+    }
+    auto prefetch_h = [&](int d) {                   // input scales: static data, may be read before the wait
+        hq[d] = make_uint4(0u, 0u, 0u, 0u);
+        if (pf_stage < n_stages && pf_stage * kStageTiles + bj < n_tiles)
+            hq[d] = __ldg(reinterpret_cast<const uint4*>(P.h + (size_t)pf_k * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
+    };
+    // MMA thread state: first segment and its output scales
+    int strip = fdiv(lo, P.div_c);
+    const int strip0 = strip;
+    int seg_end = min(n_tiles, (strip + 1) * C - lo);                       // relative to lo
+    int rt = fdiv(strip, P.div_k);
+    int k = strip - rt * G.K;
+    const int red_b = (tid >> 7) & 1, red_r = tid & 127;                   // (batch row, row) this thread reduces
+    const bool reducer = warp < kMmaWarps && red_b < NB;
+    float gval = 0.f;
+    if (warp >= kMmaWarps) {
+        if (kBuildAhead > 0) prefetch_h(0);
+    } else if (reducer && n_tiles > 0) {
+        gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
+    }
+
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- largest |x| per batch row (fp16 bit patterns order like unsigned integers once the sign is cleared)
@@ -191,76 +243,96 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     if (n_tiles == 0) return;
 
     if (warp >= kMmaWarps) {
-        // =========================== builder warps (and the copy issuer) ===========================
-        const int bl = tid - kMmaThreads;            // 0..127
-        const int j = bl >> 3, u = bl & 7;           // tile inside the stage, group of 4 columns inside the tile
-        const int tq = u & 3, half = u >> 2;
+        // =========================== builder warps (and the copy issuers) ===========================
+        const int j = bj;
         float sigma[NB][RABIT_MAX_K];
 #pragma unroll
         for (int b = 0; b < NB; ++b)
 #pragma unroll
-            for (int k = 0; k < RABIT_MAX_K; ++k) {
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
                 float inv;
-                choose_scale(S.xmax_bits[b], k < G.K ? G.hmax[k] : 0.f, sigma[b][k], inv);
+                choose_scale(S.xmax_bits[b], kk < G.K ? G.hmax[kk] : 0.f, sigma[b][kk], inv);
             }
-        long long p0 = lo + j;
-        int ct = (int)(p0 % C);
-        int k = (int)((p0 / C) % G.K);
-        for (int i = 0; i < n_stages; ++i) {
-            const int slot = i % kRing;
-            if (i >= kRing) {
-                mbar_wait(smem_u32(&S.empty[slot]), ((i / kRing) - 1) & 1, abort_flag);
-                if (tid == kMmaThreads) {
-                    const int tiles = min(kStageTiles, n_tiles - i * kStageTiles);
-                    const uint32_t bar = smem_u32(&S.full[slot]);
-                    mbar_expect_tx(bar, tiles * RABIT_TILE_BYTES);
-                    bulk_g2s(smem_u32(&S.bits[slot][0][0]), P.bits + (lo + (long long)i * kStageTiles) * RABIT_TILE_BYTES,
-                             tiles * RABIT_TILE_BYTES, bar);
-                }
+        // a queue of kBuildAhead of this pair's stages of raw inputs hides the load latency
+        uint4 xq[kBuildAhead][NB];
+        int kq[kBuildAhead];
+        auto prefetch_x = [&](int d) {
+            kq[d] = pf_k;
+#pragma unroll
+            for (int b = 0; b < NB; ++b) xq[d][b] = make_uint4(0u, 0u, 0u, 0u);
+            if (pf_stage < n_stages && pf_stage * kStageTiles + bj < n_tiles) {
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    xq[d][b] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
             }
-            const bool live = i * kStageTiles + j < n_tiles;
-            const int col = ct * RABIT_TILE_COLS + 4 * u;
-            uint2 hraw = make_uint2(0u, 0u);
-            if (live) hraw = __ldg(reinterpret_cast<const uint2*>(P.h + (size_t)k * G.N + col));
-            const float2 h01 = __half22float2(*reinterpret_cast<const __half2*>(&hraw.x));
-            const float2 h23 = __half22float2(*reinterpret_cast<const __half2*>(&hraw.y));
-            float sg[NB];
+            pf_stage += 1;
+            pf_ct += kStageTiles;
+            while (pf_ct >= C) { pf_ct -= C; pf_k = pf_k + 1 == G.K ? 0 : pf_k + 1; }
+        };
 #pragma unroll
-            for (int b = 0; b < NB; ++b) sg[b] = k == 0 ? sigma[b][0] : (k == 1 ? sigma[b][1] : sigma[b][2]);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                uint2 xraw = make_uint2(0u, 0u);
-                if (live) xraw = __ldg(reinterpret_cast<const uint2*>(P.x + (size_t)b * G.N + col));
-                const float2 x01 = __half22float2(*reinterpret_cast<const __half2*>(&xraw.x));
-                const float2 x23 = __half22float2(*reinterpret_cast<const __half2*>(&xraw.y));
-                int Tq[4];
-                Tq[0] = __float2int_rn(h01.x * x01.x * sg[b]);
-                Tq[1] = __float2int_rn(h01.y * x01.y * sg[b]);
-                Tq[2] = __float2int_rn(h23.x * x23.x * sg[b]);
-                Tq[3] = __float2int_rn(h23.y * x23.y * sg[b]);
-                long long tsum = (long long)Tq[0] + Tq[1] + Tq[2] + Tq[3];
-                tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
-                tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
-                tsum += __shfl_xor_sync(0xffffffffu, tsum, 4);
-                uint32_t X[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
-                const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
-                const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
-                uint32_t dig[4];
-                dig[0] = __byte_perm(t0, t1, 0x5410); dig[1] = __byte_perm(t0, t1, 0x7632);
-                dig[2] = __byte_perm(t2, t3, 0x5410); dig[3] = __byte_perm(t2, t3, 0x7632);
-                uint32_t* dst = reinterpret_cast<uint32_t*>(&S.table[slot][j][b * 16]) + tq * 2 + half;
-#pragma unroll
-                for (int d = 0; d < 4; ++d) dst[d * 8] = dig[d];                 // word pair index 4*d + tq
-                if (u == 0) S.sum_t[slot][j][b] = tsum;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&S.full[slot]));
-            ct += kStageTiles;
-            while (ct >= C) { ct -= C; k = k + 1 == G.K ? 0 : k + 1; }
+        for (int d = 0; d < kBuildAhead; ++d) {          // stage 0's h part was fetched before the wait
+            if (d > 0) prefetch_h(d);
+            prefetch_x(d);
         }
-        if (*abort_flag && tid == kMmaThreads) {
+
+        const bool issuer = tid == kMmaThreads;          // one lane issues the copies
+        for (int i0 = 0; i0 < n_stages; i0 += kBuildAhead) {
+#pragma unroll
+            for (int d = 0; d < kBuildAhead; ++d) {
+                const int i = i0 + d;
+                if (i >= n_stages) break;
+                const int slot = i % kRing;
+                if (i >= kRing) {
+                    mbar_wait(smem_u32(&S.empty[slot]), ((i / kRing) - 1) & 1, abort_flag);
+                    if (issuer) {
+                        const int tiles = min(kStageTiles, n_tiles - i * kStageTiles);
+                        const uint32_t bar = smem_u32(&S.full[slot]);
+                        mbar_expect_tx(bar, tiles * RABIT_TILE_BYTES);
+                        bulk_g2s(smem_u32(&S.bits[slot][0][0]), P.bits + ((size_t)lo + (size_t)i * kStageTiles) * RABIT_TILE_BYTES,
+                                 tiles * RABIT_TILE_BYTES, bar);
+                    }
+                }
+                const int kk = kq[d];
+                const uint32_t hw[4] = {hq[d].x, hq[d].y, hq[d].z, hq[d].w};
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const float sg = kk == 0 ? sigma[b][0] : (kk == 1 ? sigma[b][1] : sigma[b][2]);
+                    const uint32_t xw[4] = {xq[d][b].x, xq[d][b].y, xq[d][b].z, xq[d][b].w};
+                    int Tq[8];
+#pragma unroll
+                    for (int c2 = 0; c2 < 4; ++c2) {
+                        const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[c2]));
+                        const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[c2]));
+                        Tq[2 * c2] = __float2int_rn(hf.x * xf.x * sg);
+                        Tq[2 * c2 + 1] = __float2int_rn(hf.y * xf.y * sg);
+                    }
+                    int tsum = 0;                        // |T| < 2^28, so eight of them fit
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) tsum += Tq[c];
+                    uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][b * 16]);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
+                        const int u = 2 * bv + hlf;
+                        uint32_t X[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
+                        const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
+                        const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
+                        uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
+                        dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
+                        dst[8] = __byte_perm(t0, t1, 0x7632);
+                        dst[16] = __byte_perm(t2, t3, 0x5410);
+                        dst[24] = __byte_perm(t2, t3, 0x7632);
+                    }
+                    S.sum_t[slot][j][b][bv] = tsum;
+                }
+                prefetch_h(d);
+                prefetch_x(d);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&S.full[slot]));
+            }
+        }
+        if (*abort_flag && issuer) {
             // make sure no bulk copy is still in flight towards this CTA's shared memory
             for (int i = max(0, n_stages - kRing); i < n_stages; ++i) {
                 const long long t0 = clock64();
@@ -276,21 +348,11 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     const int gq = lane >> 2, tq = lane & 3;
     const int w = warp;
     float sig_inv[RABIT_MAX_K];               // 1 / sigma of this thread's batch row at reduction time
-    {
-        const int b = (tid >> 7) < NB ? (tid >> 7) : 0;
 #pragma unroll
-        for (int k = 0; k < RABIT_MAX_K; ++k) {
-            float sg;
-            choose_scale(S.xmax_bits[b], k < G.K ? G.hmax[k] : 0.f, sg, sig_inv[k]);
-        }
+    for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
+        float sg;
+        choose_scale(S.xmax_bits[red_b < NB ? red_b : 0], kk < G.K ? G.hmax[kk] : 0.f, sg, sig_inv[kk]);
     }
-    long long strip = lo / C;
-    int seg_end = (int)min((long long)n_tiles, (strip + 1) * C - lo);     // relative to lo
-    int k = (int)(strip % G.K);
-    int rt = (int)(strip / G.K);
-    const int red_b = tid >> 7, red_r = tid & 127;                         // this thread's (batch row, row) at reduction time
-    float gval = 0.f;
-    if (red_b < NB) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 
     int acc[8][4];
     long long sum_t[NB];
@@ -300,10 +362,21 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         for (int c = 0; c < 4; ++c) acc[p][c] = 0;
 #pragma unroll
     for (int b = 0; b < NB; ++b) sum_t[b] = 0;
+    bool red_in_use = false;
 
-    // Segment end: reduce the eight warps, scale, publish; the last contributor of the row tile finishes y.
+    // Segment end: sum the eight warps in shared memory, scale by g_k / sigma and store the
+    // partial row sums (not yet published: one fence and the arrivals follow after the last segment).
     auto segment_flush = [&]() {
-        // digits -> 2^p * sum_j b T, then sum_j T - 2 sum_j b T per row (fp32), into shared memory
+        if (red_in_use) bar_mma_warps();                                       // readers of the previous flush are done
+        red_in_use = true;
+        float st_f[NB];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {                                         // the four quarters live in lanes tq = 0..3
+            long long t = sum_t[b];
+            t += __shfl_xor_sync(0xffffffffu, t, 1);
+            t += __shfl_xor_sync(0xffffffffu, t, 2);
+            st_f[b] = __ll2float_rn(t);
+        }
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
 #pragma unroll
@@ -313,66 +386,30 @@ rabit_gemv_mma_kernel(const GemvParams P) {
                 const int b = tq >> 1;
                 if ((tq & 1) == 0 && b < NB) {
                     const float v = fmaf(65536.f, hi2, lo2);                    // 2^p * sum_j b T
-                    const float st = __ll2float_rn(b == 0 ? sum_t[0] : sum_t[NB - 1]);
+                    const float st = b == 0 ? st_f[0] : st_f[NB - 1];
                     const float scale = __int_as_float((127 + 1 - p) << 23);    // 2^(1-p)
-                    S.red[w][b][16 * p + gq + 8 * hf] = fmaf(-scale, v, st);
+                    S.red[w][b][16 * p + gq + 8 * hf] = fmaf(-scale, v, st);    // sum_j T - 2 sum_j b T
                 }
             }
         }
         bar_mma_warps();
-        if (red_b < NB) {
+        if (reducer) {
             float sum = 0.f;
 #pragma unroll
             for (int ww = 0; ww < kMmaWarps; ++ww) sum += S.red[ww][red_b][red_r];
             const float inv = k == 0 ? sig_inv[0] : (k == 1 ? sig_inv[1] : sig_inv[2]);
-            const long long seg_id = (long long)blockIdx.x + strip;
+            const size_t seg_id = (size_t)blockIdx.x + strip;
             P.partial[(seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r] = gval * (sum * inv);
         }
-        __threadfence();
-        bar_mma_warps();
-        // contributors of this row tile: for every path, the CTAs whose range meets its strip
-        int first_cta[RABIT_MAX_K], last_cta[RABIT_MAX_K];
-        unsigned int expected = 0;
-#pragma unroll
-        for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
-            first_cta[kk] = 0; last_cta[kk] = -1;
-            if (kk < G.K) {
-                const long long s0 = ((long long)rt * G.K + kk) * C;
-                first_cta[kk] = cta_of(s0, T, grid);
-                last_cta[kk] = cta_of(s0 + C - 1, T, grid);
-                expected += (unsigned int)(last_cta[kk] - first_cta[kk] + 1);
-            }
-        }
-        if (tid == 0) {
-            const unsigned int old = atomicAdd(P.counters + rt, 1u);
-            S.is_last = (old == expected - 1u);
-        }
-        bar_mma_warps();
-        if (S.is_last) {
-            __threadfence();
-            if (red_b < NB) {
-                float sum = 0.f;
-#pragma unroll
-                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-                    for (int c = first_cta[kk]; c <= last_cta[kk]; ++c) {
-                        const long long sid = (long long)c + (long long)rt * G.K + kk;
-                        sum += __ldcg(P.partial + (sid * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r);
-                    }
-                const int row = rt * RABIT_TILE_ROWS + red_r;
-                if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
-            }
-            if (tid == 0) P.counters[rt] = 0;                                   // leave the scratch clean for the next call
-        }
-        bar_mma_warps();                                                        // S.red and S.is_last are reused
     };
 
     auto next_segment = [&]() {
         strip += 1;
-        seg_end = (int)min((long long)n_tiles, (long long)seg_end + C);
+        seg_end = min(n_tiles, seg_end + C);
         k += 1;
         if (k == G.K) { k = 0; rt += 1; }
         gval = 0.f;
-        if (red_b < NB) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
+        if (reducer) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 #pragma unroll
         for (int p = 0; p < 8; ++p)
 #pragma unroll
@@ -381,41 +418,105 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         for (int b = 0; b < NB; ++b) sum_t[b] = 0;
     };
 
-    // This warp's tiles are rel = w, w + 8, ...: two per full stage, so every warp releases every full stage.
-    int cur_stage = -1;
-#pragma unroll 1
-    for (int rel = w; rel < n_tiles; rel += kMmaWarps) {
-        const int i = rel / kStageTiles, j = rel % kStageTiles;
-        const int slot = i % kRing;
-        if (i != cur_stage) {
-            if (cur_stage >= 0) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&S.empty[cur_stage % kRing]));
-            }
-            cur_stage = i;
-            mbar_wait(smem_u32(&S.full[slot]), (i / kRing) & 1, abort_flag);
-        }
-        while (rel >= seg_end) { segment_flush(); next_segment(); }
+    // This warp's tiles are rel = w, w + 8, ...: the two of a stage are taken together when both lie in
+    // the current segment (the common case), which gives the scheduler two independent chains.
+    auto one_tile = [&](int slot, int j) {
         const uint4 wv = S.bits[slot][j][lane];
         uint2 bb = make_uint2(0u, 0u);
         if (gq < 4 * NB) bb = S.table[slot][j][lane];
 #pragma unroll
-        for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][j][b];
+        for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][j][b][lane & 3];   // this lane's quarter of the tile
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             const uint32_t mask = 0x01010101u << p;
             mma_u8s8(acc[p], wv.x & mask, wv.y & mask, wv.z & mask, wv.w & mask, bb.x, bb.y);
         }
-    }
-    if (cur_stage >= 0) {
+    };
+#pragma unroll 1
+    for (int i = 0; i < n_stages; ++i) {
+        const int slot = i % kRing;
+        const int rel0 = i * kStageTiles + w, rel1 = rel0 + kMmaWarps;
+        if (rel0 >= n_tiles) break;
+        mbar_wait(smem_u32(&S.full[slot]), (i / kRing) & 1, abort_flag);
+        if (rel1 < seg_end) {
+            const uint4 wa = S.bits[slot][w][lane];
+            const uint4 wb = S.bits[slot][w + kMmaWarps][lane];
+            uint2 ba = make_uint2(0u, 0u), bb = make_uint2(0u, 0u);
+            if (gq < 4 * NB) { ba = S.table[slot][w][lane]; bb = S.table[slot][w + kMmaWarps][lane]; }
+#pragma unroll
+            for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][w][b][lane & 3] + S.sum_t[slot][w + kMmaWarps][b][lane & 3];
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                const uint32_t mask = 0x01010101u << p;
+                mma_u8s8(acc[p], wa.x & mask, wa.y & mask, wa.z & mask, wa.w & mask, ba.x, ba.y);
+            }
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                const uint32_t mask = 0x01010101u << p;
+                mma_u8s8(acc[p], wb.x & mask, wb.y & mask, wb.z & mask, wb.w & mask, bb.x, bb.y);
+            }
+        } else {
+            while (rel0 >= seg_end) { segment_flush(); next_segment(); }
+            one_tile(slot, w);
+            if (rel1 < n_tiles) {
+                while (rel1 >= seg_end) { segment_flush(); next_segment(); }
+                one_tile(slot, w + kMmaWarps);
+            }
+        }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.empty[cur_stage % kRing]));
+        if (lane == 0) mbar_arrive(smem_u32(&S.empty[slot]));
     }
     while (true) {
         segment_flush();
         if (seg_end >= n_tiles) break;
         next_segment();
     }
+
+    // ---- publish: after a CTA barrier (which orders all partial stores of the CTA before it) one
+    //      release-acquire arrival per segment; whoever completes a row tile adds its partials in a
+    //      fixed order (deterministic) and stores fp16
+    bar_mma_warps();
+    const int n_seg = strip - strip0 + 1;
+    for (int base = 0; base < n_seg; base += kMmaThreads) {
+        const int cnt = min(kMmaThreads, n_seg - base);
+        if (tid < cnt) {
+            const int rt_s = fdiv(strip0 + base + tid, P.div_k);
+            unsigned int expected = 0;
+            for (int kk = 0; kk < G.K; ++kk) {
+                const int s0 = (rt_s * G.K + kk) * C;
+                expected += (unsigned int)(cta_of(s0 + C - 1, P) - cta_of(s0, P) + 1);
+            }
+            unsigned int old;
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(P.counters + rt_s) : "memory");
+            S.flag[tid] = (old == expected - 1u) ? 1 : 0;
+        }
+        bar_mma_warps();
+        for (int q = 0; q < cnt; ++q) {
+            if (!S.flag[q]) continue;
+            const int rt_s = fdiv(strip0 + base + q, P.div_k);
+            if (reducer) {
+                float sum = 0.f;
+                for (int kk = 0; kk < G.K; ++kk) {
+                    const int s0 = (rt_s * G.K + kk) * C;
+                    const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
+                    const float* src = P.partial + (((size_t)c0 + (size_t)rt_s * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+                    for (int c = c0; c <= c1; c += 8) {                       // eight loads in flight, summed in order
+                        float v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) v[u] = c + u <= c1 ? __ldcg(src + (size_t)u * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS) : 0.f;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) sum += v[u];
+                        src += (size_t)8 * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+                    }
+                }
+                const int row = rt_s * RABIT_TILE_ROWS + red_r;
+                if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
+            }
+            if (tid == 0) P.counters[rt_s] = 0;                                 // leave the scratch clean for the next call
+        }
+        bar_mma_warps();                                                        // S.flag is reused
+    }
+    if (*abort_flag && tid == 0) atomicExch(P.status, 1u);
 }
 
 }  // namespace
@@ -458,9 +559,15 @@ cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, 
     P.partial = L.d_partial;
     P.counters = L.d_counters;
     P.status = L.d_status;
-    P.n_tiles = (long long)L.geom.n_rt * L.geom.K * L.geom.n_ct;
-    int grid = L.sm_count > 0 ? L.sm_count : 148;
+    P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
+    int grid = 2 * (L.sm_count > 0 ? L.sm_count : 148);      // two co-resident CTAs per SM
     if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
-    if ((long long)grid > P.n_tiles) grid = (int)P.n_tiles;
+    if (grid > P.n_tiles) grid = P.n_tiles;
+    P.q = P.n_tiles / grid;
+    P.r = P.n_tiles % grid;
+    P.div_c = make_fastdiv((unsigned int)L.geom.n_ct);
+    P.div_k = make_fastdiv((unsigned int)L.geom.K);
+    P.div_q = make_fastdiv((unsigned int)P.q);
+    P.div_q1 = make_fastdiv((unsigned int)P.q + 1u);
     return batch == 1 ? launch_nb<1>(P, grid, stream) : launch_nb<2>(P, grid, stream);
 }
