@@ -213,6 +213,7 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     const int red_b = (tid >> 7) & 1, red_r = tid & 127;                   // (batch row, row) this thread reduces
     const bool reducer = warp < kMmaWarps && red_b < NB;
     float gval = 0.f;
+    if (tid == 0 && n_tiles > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.counters + rt));
     if (warp >= kMmaWarps) {
         if (kBuildAhead > 0) prefetch_h(0);
     } else if (reducer && n_tiles > 0) {
@@ -495,19 +496,37 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             if (!S.flag[q]) continue;
             const int rt_s = fdiv(strip0 + base + q, P.div_k);
             if (reducer) {
-                float sum = 0.f;
-                for (int kk = 0; kk < G.K; ++kk) {
-                    const int s0 = (rt_s * G.K + kk) * C;
-                    const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
-                    const float* src = P.partial + (((size_t)c0 + (size_t)rt_s * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
-                    for (int c = c0; c <= c1; c += 8) {                       // eight loads in flight, summed in order
-                        float v[8];
+                // contributions are listed path by path, CTA by CTA; up to 8 per path are loaded at once
+                const float* src[RABIT_MAX_K];
+                int cnt_k[RABIT_MAX_K];
+                bool small = true;
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) v[u] = c + u <= c1 ? __ldcg(src + (size_t)u * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS) : 0.f;
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) sum += v[u];
-                        src += (size_t)8 * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+                for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
+                    src[kk] = P.partial; cnt_k[kk] = 0;
+                    if (kk < G.K) {
+                        const int s0 = (rt_s * G.K + kk) * C;
+                        const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
+                        src[kk] = P.partial + (((size_t)c0 + (size_t)rt_s * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+                        cnt_k[kk] = c1 - c0 + 1;
+                        small = small && cnt_k[kk] <= 8;
                     }
+                }
+                constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+                float sum = 0.f;
+                if (small) {
+                    float v[RABIT_MAX_K][8];
+#pragma unroll
+                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) v[kk][u] = u < cnt_k[kk] ? __ldcg(src[kk] + u * kStride) : 0.f;
+#pragma unroll
+                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) sum += v[kk][u];
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                        for (int c = 0; c < cnt_k[kk]; ++c) sum += __ldcg(src[kk] + c * kStride);
                 }
                 const int row = rt_s * RABIT_TILE_ROWS + red_r;
                 if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
