@@ -5,8 +5,8 @@ library image can be compared byte for byte.  The paper fixes only the sign -> b
 (Appendix "Weight Packing": +1 -> 0, -1 -> 1); the arrangement below is this build's.
 
 Image = header (256 B) | sign tiles | g fp16 [K][Mp] | h fp16 [K][N] | fp32 partial scratch
-[n_rt*K + max_grid][partial_batch][128] | u32 counters [n_rt] + one status word; every
-section starts on a 256-byte boundary; padding, scratch, counters and status are zero.
+[n_rt*K + max_grid][partial_batch][128] | u32 flags [n_rt*K + max_grid] + one status word; every
+section starts on a 256-byte boundary; padding, scratch, flags and status are zero.
 Mp = M rounded up to 128; padded signs are +1 (bit 0), padded scales 0; N is a multiple of
 32 and is not padded.  The header also records max_j |h_k[j]| per path as an fp32 bit
 pattern (the kernels derive their fixed-point scale from it).
@@ -36,7 +36,7 @@ PARTIAL_BATCH = 4
 _HEADER_FMT = "<16I6Q"
 _HEADER_KEYS = ["magic", "version", "K", "M", "N", "Mp", "n_rt", "n_ct", "max_grid", "partial_batch",
                 "hmax0", "hmax1", "hmax2", "hmax3", "reserved0", "reserved1",
-                "off_bits", "off_g", "off_h", "off_partial", "off_counters", "total_bytes"]
+                "off_bits", "off_g", "off_h", "off_partial", "off_flags", "total_bytes"]
 
 
 def _align256(v: int) -> int:
@@ -52,7 +52,7 @@ def geometry(K: int, M: int, N: int) -> dict:
     geo["off_g"] = off; off = _align256(off + K * Mp * 2)
     geo["off_h"] = off; off = _align256(off + K * N * 2)
     geo["off_partial"] = off; off = _align256(off + (n_rt * K + MAX_GRID) * PARTIAL_BATCH * TILE_ROWS * 4)
-    geo["off_counters"] = off; off = _align256(off + n_rt * 4 + 4)
+    geo["off_flags"] = off; off = _align256(off + (n_rt * K + MAX_GRID) * 4 + 4)
     geo["total_bytes"] = off
     return geo
 
@@ -61,7 +61,7 @@ def header_bytes(geo: dict, hmax_bits) -> bytes:
     hm = list(hmax_bits) + [0] * (4 - len(hmax_bits))
     head = struct.pack(_HEADER_FMT, MAGIC, VERSION, geo["K"], geo["M"], geo["N"], geo["Mp"], geo["n_rt"], geo["n_ct"],
                        MAX_GRID, PARTIAL_BATCH, hm[0], hm[1], hm[2], hm[3], 0, 0,
-                       geo["off_bits"], geo["off_g"], geo["off_h"], geo["off_partial"], geo["off_counters"],
+                       geo["off_bits"], geo["off_g"], geo["off_h"], geo["off_partial"], geo["off_flags"],
                        geo["total_bytes"])
     return head + bytes(HEADER_BYTES - len(head))
 

@@ -71,8 +71,8 @@ extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint1
     L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
     L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
     L->d_partial = (float*)(L->dev_base + hdr.off_partial);
-    L->d_counters = (unsigned int*)(L->dev_base + hdr.off_counters);
-    L->d_status = L->d_counters + G.n_rt;
+    L->d_flags = (unsigned int*)(L->dev_base + hdr.off_flags);
+    L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
     *out = L;
     return RABIT_OK;
 }

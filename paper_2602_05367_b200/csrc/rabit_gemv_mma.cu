@@ -27,9 +27,11 @@
 //   * Eight MMA warps take the tiles of a stage round-robin: one 128-bit shared-memory read
 //     of weights, one 64-bit read of digits, 32 ANDs and 8 MMAs per 4096 weights.
 //   * A segment is the part of the CTA range inside one (row tile, path) strip.  At a
-//     segment end the warps are summed in shared memory, scaled by g_k / sigma and written
-//     to a per-layer fp32 partial buffer; the CTA whose arrival completes a row tile adds
-//     the partials in a fixed order (deterministic) and stores fp16.
+//     segment end the warps are summed in shared memory, scaled by g_k / sigma, written to
+//     a per-layer fp32 partial buffer and published with a release store of a flag.  The
+//     CTA that owns the last tile of a row tile finishes it: it acquires the flags of the
+//     other contributors (all of them CTAs with a lower index, so the waits cannot form a
+//     cycle), adds the partials in a fixed order (deterministic) and stores fp16.
 // Every wait in the kernel is bounded; a wait that runs out sets a status word and the
 // kernel drains and returns (results are then invalid, the context stays usable).
 #include <cuda_fp16.h>
@@ -71,11 +73,11 @@ struct GemvParams {
     const __half* x;
     __half* y;
     float* partial;          // [n_rt*K + grid][RABIT_PARTIAL_BATCH][128]
-    unsigned int* counters;  // [n_rt]
+    unsigned int* flags;     // [n_rt*K + grid]: segment (CTA c, strip s) publishes its partial under index c + s
     unsigned int* status;
     int n_tiles;             // n_rt * K * n_ct (< 2^31)
     int q, r;                // n_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
-    FastDiv div_c, div_k, div_q, div_q1;   // by n_ct, K, q, q + 1
+    FastDiv div_c, div_k, div_kc, div_q, div_q1;   // by n_ct, K, K * n_ct, q, q + 1
 };
 
 template <int NB>
@@ -88,7 +90,6 @@ struct __align__(128) Smem {
     unsigned long long empty[kRing];
     unsigned int xmax_bits[NB];
     int abort_flag;
-    int flag[kMmaThreads];                              // per segment: did this CTA complete the row tile
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -206,14 +207,12 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     };
     // MMA thread state: first segment and its output scales
     int strip = fdiv(lo, P.div_c);
-    const int strip0 = strip;
     int seg_end = min(n_tiles, (strip + 1) * C - lo);                       // relative to lo
     int rt = fdiv(strip, P.div_k);
     int k = strip - rt * G.K;
     const int red_b = (tid >> 7) & 1, red_r = tid & 127;                   // (batch row, row) this thread reduces
     const bool reducer = warp < kMmaWarps && red_b < NB;
     float gval = 0.f;
-    if (tid == 0 && n_tiles > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.counters + rt));
     if (warp >= kMmaWarps) {
         if (kBuildAhead > 0) prefetch_h(0);
     } else if (reducer && n_tiles > 0) {
@@ -363,13 +362,12 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         for (int c = 0; c < 4; ++c) acc[p][c] = 0;
 #pragma unroll
     for (int b = 0; b < NB; ++b) sum_t[b] = 0;
-    bool red_in_use = false;
+    const int me = blockIdx.x;
+    const int KC = G.K * C;
 
-    // Segment end: sum the eight warps in shared memory, scale by g_k / sigma and store the
-    // partial row sums (not yet published: one fence and the arrivals follow after the last segment).
+    // Segment end: sum the eight warps in shared memory, scale by g_k / sigma, store the partial row
+    // sums and publish them (unless this CTA is the one that will finish the row tile itself).
     auto segment_flush = [&]() {
-        if (red_in_use) bar_mma_warps();                                       // readers of the previous flush are done
-        red_in_use = true;
         float st_f[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) {                                         // the four quarters live in lanes tq = 0..3
@@ -394,14 +392,17 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             }
         }
         bar_mma_warps();
+        const int seg_id = me + strip;
         if (reducer) {
             float sum = 0.f;
 #pragma unroll
             for (int ww = 0; ww < kMmaWarps; ++ww) sum += S.red[ww][red_b][red_r];
             const float inv = k == 0 ? sig_inv[0] : (k == 1 ? sig_inv[1] : sig_inv[2]);
-            const size_t seg_id = (size_t)blockIdx.x + strip;
-            P.partial[(seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r] = gval * (sum * inv);
+            P.partial[((size_t)seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r] = gval * (sum * inv);
         }
+        bar_mma_warps();                                                        // partial stores ordered before the release; S.red free again
+        if (tid == 0 && cta_of((rt + 1) * KC - 1, P) != me)
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(P.flags + seg_id), "r"(1u) : "memory");
     };
 
     auto next_segment = [&]() {
@@ -473,67 +474,65 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         next_segment();
     }
 
-    // ---- publish: after a CTA barrier (which orders all partial stores of the CTA before it) one
-    //      release-acquire arrival per segment; whoever completes a row tile adds its partials in a
-    //      fixed order (deterministic) and stores fp16
-    bar_mma_warps();
-    const int n_seg = strip - strip0 + 1;
-    for (int base = 0; base < n_seg; base += kMmaThreads) {
-        const int cnt = min(kMmaThreads, n_seg - base);
-        if (tid < cnt) {
-            const int rt_s = fdiv(strip0 + base + tid, P.div_k);
-            unsigned int expected = 0;
-            for (int kk = 0; kk < G.K; ++kk) {
-                const int s0 = (rt_s * G.K + kk) * C;
-                expected += (unsigned int)(cta_of(s0 + C - 1, P) - cta_of(s0, P) + 1);
+    // ---- finish the row tiles whose last tile this CTA owns: wait (bounded) for the flags of the other
+    //      contributors, add all partials in a fixed order, store fp16, clear the flags for the next call
+    for (int rt_f = fdiv(lo, P.div_kc); (rt_f + 1) * KC - 1 < lo + n_tiles; ++rt_f) {
+        // contributors: for every path kk the CTAs c0..c1 whose range meets strip (rt_f, kk)
+        int c0k[RABIT_MAX_K], cntk[RABIT_MAX_K];
+        int total = 0;
+        bool small = true;
+#pragma unroll
+        for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
+            c0k[kk] = 0; cntk[kk] = 0;
+            if (kk < G.K) {
+                const int s0 = (rt_f * G.K + kk) * C;
+                c0k[kk] = cta_of(s0, P);
+                cntk[kk] = cta_of(s0 + C - 1, P) - c0k[kk] + 1;
+                total += cntk[kk];
+                small = small && cntk[kk] <= 8;
             }
-            unsigned int old;
-            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(P.counters + rt_s) : "memory");
-            S.flag[tid] = (old == expected - 1u) ? 1 : 0;
+        }
+        for (int e = tid; e < total; e += kMmaThreads) {
+            int kk = 0, c = e;
+            while (c >= cntk[kk]) { c -= cntk[kk]; ++kk; }
+            c += c0k[kk];
+            if (c == me) continue;
+            const unsigned int* f = P.flags + (c + rt_f * G.K + kk);
+            unsigned int v;
+            const long long t0 = clock64();
+            while (true) {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                if (v) break;
+                if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
+            }
+            *const_cast<unsigned int*>(f) = 0u;                                   // leave the scratch clean for the next call
         }
         bar_mma_warps();
-        for (int q = 0; q < cnt; ++q) {
-            if (!S.flag[q]) continue;
-            const int rt_s = fdiv(strip0 + base + q, P.div_k);
-            if (reducer) {
-                // contributions are listed path by path, CTA by CTA; up to 8 per path are loaded at once
-                const float* src[RABIT_MAX_K];
-                int cnt_k[RABIT_MAX_K];
-                bool small = true;
+        if (reducer) {
+            constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+            const float* src[RABIT_MAX_K];
 #pragma unroll
-                for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
-                    src[kk] = P.partial; cnt_k[kk] = 0;
-                    if (kk < G.K) {
-                        const int s0 = (rt_s * G.K + kk) * C;
-                        const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
-                        src[kk] = P.partial + (((size_t)c0 + (size_t)rt_s * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
-                        cnt_k[kk] = c1 - c0 + 1;
-                        small = small && cnt_k[kk] <= 8;
-                    }
-                }
-                constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
-                float sum = 0.f;
-                if (small) {
-                    float v[RABIT_MAX_K][8];
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                src[kk] = P.partial + (((size_t)c0k[kk] + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+            float sum = 0.f;
+            if (small) {
+                float v[RABIT_MAX_K][8];
 #pragma unroll
-                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) v[kk][u] = u < cnt_k[kk] ? __ldcg(src[kk] + u * kStride) : 0.f;
+                    for (int u = 0; u < 8; ++u) v[kk][u] = u < cntk[kk] ? __ldcg(src[kk] + u * kStride) : 0.f;
 #pragma unroll
-                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) sum += v[kk][u];
-                } else {
+                    for (int u = 0; u < 8; ++u) sum += v[kk][u];
+            } else {
 #pragma unroll
-                    for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-                        for (int c = 0; c < cnt_k[kk]; ++c) sum += __ldcg(src[kk] + c * kStride);
-                }
-                const int row = rt_s * RABIT_TILE_ROWS + red_r;
-                if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
+                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                    for (int c = 0; c < cntk[kk]; ++c) sum += __ldcg(src[kk] + c * kStride);
             }
-            if (tid == 0) P.counters[rt_s] = 0;                                 // leave the scratch clean for the next call
+            const int row = rt_f * RABIT_TILE_ROWS + red_r;
+            if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
         }
-        bar_mma_warps();                                                        // S.flag is reused
     }
     if (*abort_flag && tid == 0) atomicExch(P.status, 1u);
 }
@@ -576,7 +575,7 @@ cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, 
     P.x = (const __half*)x;
     P.y = (__half*)y;
     P.partial = L.d_partial;
-    P.counters = L.d_counters;
+    P.flags = L.d_flags;
     P.status = L.d_status;
     P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
     int grid = 2 * (L.sm_count > 0 ? L.sm_count : 148);      // two co-resident CTAs per SM
@@ -586,6 +585,7 @@ cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, 
     P.r = P.n_tiles % grid;
     P.div_c = make_fastdiv((unsigned int)L.geom.n_ct);
     P.div_k = make_fastdiv((unsigned int)L.geom.K);
+    P.div_kc = make_fastdiv((unsigned int)(L.geom.K * L.geom.n_ct));
     P.div_q = make_fastdiv((unsigned int)P.q);
     P.div_q1 = make_fastdiv((unsigned int)P.q + 1u);
     return batch == 1 ? launch_nb<1>(P, grid, stream) : launch_nb<2>(P, grid, stream);

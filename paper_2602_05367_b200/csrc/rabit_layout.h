@@ -51,7 +51,7 @@ struct RabitHeader {            // first 256 bytes of a packed image (little end
     uint32_t partial_batch;     // RABIT_PARTIAL_BATCH at pack time
     uint32_t hmax_bits[4];      // fp32 bit pattern of max_j |h_k[j]| per path (0 for unused paths)
     uint32_t reserved[2];
-    uint64_t off_bits, off_g, off_h, off_partial, off_counters, total_bytes;
+    uint64_t off_bits, off_g, off_h, off_partial, off_flags, total_bytes;
     uint8_t pad[RABIT_HEADER_BYTES - 16 * 4 - 6 * 8];
 };
 

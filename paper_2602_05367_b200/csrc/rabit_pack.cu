@@ -54,7 +54,7 @@ void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr) {
     hdr->off_g = off;        off = rabit_align256(off + (size_t)G.K * G.Mp * 2);
     hdr->off_h = off;        off = rabit_align256(off + (size_t)G.K * G.N * 2);
     hdr->off_partial = off;  off = rabit_align256(off + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID) * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS * 4);
-    hdr->off_counters = off; off = rabit_align256(off + (size_t)G.n_rt * 4 + 4);   // + one status word
+    hdr->off_flags = off;    off = rabit_align256(off + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID) * 4 + 4);   // + one status word
     hdr->total_bytes = off;
 }
 
