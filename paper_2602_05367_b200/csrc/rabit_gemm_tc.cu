@@ -1,4 +1,347 @@
-// placeholder until the tcgen05 GEMM lands
+// Large-batch form of the layer on the tcgen05 tensor cores (batch > 16).
+//
+//   y[b][i] = sum_k g_k[i] * sum_j (B_k[i][j] * h_k[j]) * x[b][j]                       (Section 4.1, Eq. 2)
+//
+// For many activation rows the layer is a dense contraction.  Per path k the A operand is the
+// sign tile with the input scale folded in, A_k[i][j] = +-h_k[j]: an fp16 value with its sign
+// bit flipped by the weight bit, so the expansion is exact.  The B operand is x itself (fp16,
+// loaded by TMA, shared by all paths), products are exact in fp32 and accumulate in fp32 in
+// tensor memory; the epilogue applies g_k, adds the paths and rounds once to fp16.
+//
+// One CTA per SM, persistent over output tiles of 128 weight rows x 256 batch rows:
+//   warp 0      producer: per 64-column step, one TMA tile of x (128B swizzle) plus bulk copies of
+//               the packed sign tiles and the h slices of that step, into a 3-stage ring
+//   warp 1      allocates tensor memory, issues tcgen05.mma (M=128, N=256, K=16, kind::f16) for every
+//               path into that path's accumulator, commits stages back to the producer
+//   warps 2..9  expand packed signs to +-h fp16 in the canonical K-major 128B-swizzled layout, then
+//               (same warps) read the accumulators with tcgen05.ld for the epilogue
+// Every wait is bounded; on a time-out the CTA sets the status word, skips the remaining waits,
+// frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
 #include "rabit_internal.h"
-bool rabit_gemm_tc_supports(const rabit_layer&, int) { return false; }
-cudaError_t rabit_launch_gemm_tc(const rabit_layer&, const void*, void*, int, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kTileM = 128;                 // weight rows per output tile
+constexpr int kTileB = 256;                 // batch rows per output tile (MMA N)
+constexpr int kStepCols = 64;               // input columns per pipeline step (128 bytes of fp16: one swizzle row)
+constexpr int kStages = 3;
+constexpr int kMaxPaths = 2;                // accumulators of 256 columns: 2 x 256 = the 512 columns of tensor memory
+constexpr int kExpandWarps = 8;
+constexpr int kThreads = (2 + kExpandWarps) * 32;
+constexpr long long kWaitLimitCycles = 1LL << 31;
+
+struct __align__(1024) Stage {
+    __half a[kMaxPaths][kTileM * kStepCols];          // 2 x 16 KB, +-h, swizzled
+    __half x[kTileB * kStepCols];                     // 32 KB, swizzled by TMA
+    uint4 bits[kMaxPaths][2][32];                     // packed sign tiles: 2 column tiles per step per path
+    __half h[kMaxPaths][kStepCols];
+};
+
+struct Smem {
+    Stage stage[kStages];
+    unsigned long long full[kStages];                 // TMA bytes landed (x, bits, h)
+    unsigned long long a_ready[kStages];              // expanders done
+    unsigned long long empty[kStages];                // MMAs that read the stage retired
+    unsigned long long acc_ready;                     // all MMAs of the tile retired
+    unsigned long long acc_empty;                     // epilogue has read the accumulators
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct GemmParams {
+    RabitGeom G;
+    const unsigned char* bits;
+    const __half* g;
+    const __half* h;
+    __half* y;
+    unsigned int* status;
+    int batch;
+    int n_bt;                                         // batch tiles
+    int n_tiles;                                      // n_rt * n_bt
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return; }
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart; descriptor version 1.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    uint64_t d = (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset
+    d |= (uint64_t)1 << 46;                        // descriptor version
+    d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B fp16, both K-major, N = 256, M = 128.
+__device__ __forceinline__ uint32_t umma_idesc() {
+    return (1u << 4) | ((uint32_t)(kTileB >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_map) {
+    extern __shared__ unsigned char smem_raw[];
+    // the swizzled operand tiles need 1024-byte alignment; the launch reserves the slack
+    Smem& S = *reinterpret_cast<Smem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    const RabitGeom& G = P.G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = G.K;
+    const int n_steps = (G.N + kStepCols - 1) / kStepCols;        // N % 32 == 0: the last step may hold one column tile only
+    volatile int* abort_flag = &S.abort_flag;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&S.full[s]), 1);
+            mbar_init(smem_u32(&S.a_ready[s]), kExpandWarps);
+            mbar_init(smem_u32(&S.empty[s]), 1);
+        }
+        mbar_init(smem_u32(&S.acc_ready), 1);
+        mbar_init(smem_u32(&S.acc_empty), kExpandWarps);
+        S.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {                                            // one warp allocates all 512 columns of tensor memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&S.tmem_base)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = S.tmem_base;
+
+    if (warp == 0) {
+        // ===================================== producer =====================================
+        if (lane == 0) {
+            int it = 0;                                          // global step counter of this CTA
+            for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x) {
+                const int rt = t / P.n_bt, bt = t % P.n_bt;
+                for (int s = 0; s < n_steps; ++s, ++it) {
+                    const int slot = it % kStages;
+                    if (it >= kStages) mbar_wait(smem_u32(&S.empty[slot]), ((it / kStages) - 1) & 1, abort_flag);
+                    Stage& st = S.stage[slot];
+                    const int cts = min(2, G.n_ct - 2 * s);      // column tiles in this step
+                    const uint32_t bar = smem_u32(&S.full[slot]);
+                    const uint32_t bytes = (uint32_t)(kTileB * kStepCols * 2) + (uint32_t)K * cts * (RABIT_TILE_BYTES + RABIT_TILE_COLS * 2);
+                    mbar_expect_tx(bar, bytes);
+                    tma_load_2d(smem_u32(st.x), &x_map, s * kStepCols, bt * kTileB, bar);
+                    for (int k = 0; k < K; ++k) {
+                        bulk_g2s(smem_u32(&st.bits[k][0][0]), P.bits + rabit_tile_pos(G, rt, k, 2 * s) * RABIT_TILE_BYTES,
+                                 cts * RABIT_TILE_BYTES, bar);
+                        bulk_g2s(smem_u32(&st.h[k][0]), P.h + (size_t)k * G.N + (size_t)s * kStepCols, cts * RABIT_TILE_COLS * 2, bar);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================================== MMA issuer =====================================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc();
+            int it = 0, tile_i = 0;
+            for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
+                if (tile_i > 0) mbar_wait(smem_u32(&S.acc_empty), (tile_i - 1) & 1, abort_flag);   // epilogue has drained the accumulators
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int s = 0; s < n_steps; ++s, ++it) {
+                    const int slot = it % kStages;
+                    mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
+                    mbar_wait(smem_u32(&S.a_ready[slot]), (it / kStages) & 1, abort_flag);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    Stage& st = S.stage[slot];
+                    const int ksub = min(2, G.n_ct - 2 * s) * 2;                                   // MMAs of K = 16 in this step (2 per column tile)
+                    const uint64_t bdesc = umma_desc(smem_u32(st.x));
+                    for (int k = 0; k < K; ++k) {
+                        const uint64_t adesc = umma_desc(smem_u32(st.a[k]));
+                        for (int kk = 0; kk < ksub; ++kk)
+                            umma_f16(tmem_base + (uint32_t)k * kTileB, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc,
+                                     (s > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&S.empty[slot]));                                         // frees the stage when these MMAs retire
+                }
+                umma_commit(smem_u32(&S.acc_ready));
+            }
+        }
+    } else {
+        // ============================ expanders, then epilogue ============================
+        const int e = warp - 2;                               // 0..7
+        const int et = e * 32 + lane;                         // 0..255
+        const int quarter = warp & 3;                         // tensor-memory lanes this warp may read: 32*quarter .. +31
+        const int col_half = e >> 2;                          // which 128 of the 256 batch columns this warp drains
+        int it = 0, tile_i = 0;
+        for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
+            const int rt = t / P.n_bt, bt = t % P.n_bt;
+            for (int s = 0; s < n_steps; ++s, ++it) {
+                const int slot = it % kStages;
+                mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
+                Stage& st = S.stage[slot];
+                const int cts = min(2, G.n_ct - 2 * s);
+                // packed words of the step: [path][column tile][lane][word a]; 256 threads take them round-robin
+                for (int wi = et; wi < K * 2 * 128; wi += kExpandWarps * 32) {
+                    const int k = wi >> 8, ct2 = (wi >> 7) & 1, l = (wi >> 2) & 31, a = wi & 3;
+                    const int gq = l >> 2, tq = l & 3;
+                    uint32_t w = 0;
+                    uint2 hv = make_uint2(0u, 0u);
+                    if (ct2 < cts) {
+                        w = reinterpret_cast<const uint32_t*>(&st.bits[k][ct2][l])[a];
+                        hv = *reinterpret_cast<const uint2*>(&st.h[k][32 * ct2 + 16 * (a >> 1) + 4 * tq]);
+                    }
+                    // columns 32*ct2 + 16*(a>>1) + 4*tq + c (c = 0..3) = bytes 0..7 of 16-byte chunk number
+                    // 4*ct2 + 2*(a>>1) + (tq>>1) in the row, second half if tq is odd; rows 16*p + gq + 8*(a&1)
+                    const int chunk = 4 * ct2 + 2 * (a >> 1) + (tq >> 1);
+                    unsigned char* base = reinterpret_cast<unsigned char*>(st.a[k]) + (gq + 8 * (a & 1)) * 128 + ((chunk ^ gq) << 4) + 8 * (tq & 1);
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        const uint32_t sh = w << (7 - p);                                  // bit p of every byte -> bit 7
+                        const uint32_t s01 = __byte_perm(sh, 0u, 0x1404);                  // bytes [0, c0, 0, c1]
+                        const uint32_t s23 = __byte_perm(sh, 0u, 0x3424);                  // bytes [0, c2, 0, c3]
+                        uint2 o;
+                        o.x = hv.x ^ (s01 & 0x80008000u);                                  // flip the fp16 sign where the weight is -1
+                        o.y = hv.y ^ (s23 & 0x80008000u);
+                        *reinterpret_cast<uint2*>(base + p * 16 * 128) = o;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");              // generic-proxy writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&S.a_ready[slot]));
+            }
+            // ---- epilogue of this tile
+            mbar_wait(smem_u32(&S.acc_ready), tile_i & 1, abort_flag);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int row = rt * kTileM + quarter * 32 + lane;
+            float gk[kMaxPaths];
+#pragma unroll
+            for (int k = 0; k < kMaxPaths; ++k) gk[k] = (k < K && row < G.Mp) ? __half2float(P.g[(size_t)k * G.Mp + row]) : 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                const int col = col_half * 128 + c0;
+                uint32_t d0[32], d1[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, d0);
+                if (K > 1) tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(kTileB + col), d1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    float v = gk[0] * __uint_as_float(d0[c]);
+                    if (K > 1) v = fmaf(gk[1], __uint_as_float(d1[c]), v);
+                    const int b = bt * kTileB + col + c;
+                    if (b < P.batch && row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(v);
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&S.acc_empty));
+        }
+    }
+
+    // ---- teardown: everyone meets, then the allocating warp frees the tensor memory
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+    if (tid == 0 && *abort_flag) atomicExch(P.status, 1u);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool rabit_gemm_tc_supports(const rabit_layer& L, int batch) {
+    return batch > RABIT_MAX_GEMV_BATCH && L.geom.K <= kMaxPaths && encode_tiled_fn() != nullptr;
+}
+
+cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)L.geom.N, (cuuint64_t)batch};
+    const cuuint64_t strides[1] = {(cuuint64_t)L.geom.N * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kStepCols, (cuuint32_t)kTileB};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+
+    GemmParams P;
+    P.G = L.geom;
+    P.bits = reinterpret_cast<const unsigned char*>(L.d_bits);
+    P.g = (const __half*)L.d_g;
+    P.h = (const __half*)L.d_h;
+    P.y = (__half*)y;
+    P.status = L.d_status;
+    P.batch = batch;
+    P.n_bt = (batch + kTileB - 1) / kTileB;
+    P.n_tiles = L.geom.n_rt * P.n_bt;
+    static bool attr_done = false;
+    const size_t smem = sizeof(Smem) + 1024;                       // slack for the 1024-byte alignment of the stages
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    int grid = L.sm_count > 0 ? L.sm_count : 148;
+    if (grid > P.n_tiles) grid = P.n_tiles;
+    rabit_gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(P, map);
+    return cudaGetLastError();
+}
