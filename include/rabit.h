@@ -113,6 +113,35 @@ RABIT_API size_t rabit_stage_bytes(const rabit_layer* layer, int batch);
 RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, void* y_host, int batch,
                       void* dev_stage, size_t dev_stage_bytes, void* stream);
 
+/*
+ * The batch 1..16 layer call for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a host that hands out a
+ * fixed memory budget at start-up, in a real-time loop where an allocation may block or
+ * synchronise the device, or in a plug-in that is given weight, input and output buffers but no
+ * allocator.  rabit_linear keeps its reduction scratch inside the caller-allocated packed image;
+ * a caller that received only the weights section of an image (or a read-only mapping of it) has
+ * nowhere to put that scratch.  This entry point uses a fixed 4 MiB device array that is part of
+ * the library instead (every GPU that loads the library holds these 4 MiB until the process exits).
+ *
+ *   layer, x, y, batch, stream   as rabit_linear, with 1 <= batch <= 16; the layer's device must be
+ *                                the current device.
+ * Limits and rules:
+ *   - The scratch a layer needs is (K * ceil(M/128) + 320) * 2052 bytes, rounded up; a layer that
+ *     needs more than the 4 MiB array is refused with RABIT_UNSUPPORTED_SHAPE and a message that
+ *     states both sizes (K = 2 layers up to about M = 110,000 rows fit).
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on a
+ *     device looks up the device address of the array (cudaGetSymbolAddress); make that first
+ *     call before any stream capture begins.
+ *   - All calls, for all layers, share the one array.  Each call clears the part that must start
+ *     at zero (a memset enqueued on `stream` ahead of the kernel).  Two calls that overlap on the
+ *     GPU (different streams, or one stream per thread) race on it and give wrong results: keep
+ *     all uses of this entry point on one stream, or serialise them yourself.
+ * Results equal those of rabit_linear (same kernel, same summation order).
+ */
+RABIT_API int rabit_linear_static_scratch(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
+
 /* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
 RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
                  void* stream);

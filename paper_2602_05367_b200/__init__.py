@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     rabit_pack,
     rabit_linear,
     rabit_linear_host,
+    rabit_linear_static_scratch,
     rabit_free,
     last_error,
 )

@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     lib.rabit_stage_bytes.argtypes = [_c_void_p, _c_int]
     lib.rabit_linear_host.restype = _c_int
     lib.rabit_linear_host.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]
+    lib.rabit_linear_static_scratch.restype = _c_int
+    lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
     lib.rabit_unpack.restype = _c_int
     lib.rabit_unpack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p]
     for name in ("rabit_layer_K", "rabit_layer_M", "rabit_layer_N"):
@@ -216,6 +218,25 @@ def rabit_linear_host(layer: RabitLayer, x_host, y_host, stream: Optional[int] =
     _check(_lib.rabit_linear_host(layer.handle, _c_void_p(x_host.data_ptr()), _c_void_p(y_host.data_ptr()), batch,
                                   _c_void_p(layer._stage.data_ptr()), need, _c_void_p(st)))
     return y_host
+
+
+def rabit_linear_static_scratch(layer: RabitLayer, x, y, stream: Optional[int] = None):
+    """rabit_linear for batch 1..16 that keeps its reduction scratch in the library's own fixed
+    4 MiB device array, so nothing is allocated for the call (the caller passes x and y).  All
+    calls share that array: keep them on one stream."""
+    import torch
+
+    if x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA float16 tensor")
+    if y.dtype != torch.float16 or not y.is_cuda or not y.is_contiguous():
+        raise ValueError("y must be a contiguous CUDA float16 tensor")
+    batch = 1 if x.dim() == 1 else x.shape[0]
+    if x.numel() != batch * layer.N or y.numel() != batch * layer.M:
+        raise ValueError("x / y sizes do not match the layer")
+    st = torch.cuda.current_stream(x.device).cuda_stream if stream is None else stream
+    with torch.cuda.device(x.device):
+        _check(_lib.rabit_linear_static_scratch(layer.handle, _c_void_p(x.data_ptr()), _c_void_p(y.data_ptr()), batch, _c_void_p(st)))
+    return y
 
 
 def rabit_free(layer: RabitLayer) -> None:
