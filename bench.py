@@ -307,6 +307,94 @@ def cpu_baseline(sample_projections: int = 7, repeats: int = 1) -> dict:
             "sample": "decoder-layer copy 0, its %d projections once each, batch 1 (float64: unpack signs, dense W, product)" % len(shapes)}
 
 
+def bench_cases(args) -> dict:
+    """Extra workloads (not the default line): one (shape, batch) case at a time, rotating over enough
+    distinct copies of the layer to exceed L2, CUDA-graph replay, CUDA-event timing.
+      gemm70b : 70B-shaped layers at batch 512 (tensor-core GEMM), roofline = measured bf16 TFLOP/s
+      gemv70b : the same layers at batch 1 (HBM roofline)
+      sweep8b : Llama-3-8B shapes at batch 1,2,4,8,16 (HBM roofline per batch)"""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from synth import llama3_8b_layer_shapes, llama_70b_layer_shapes, make_layer, make_x
+
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    if args.workload == "sweep8b":
+        seen, shapes = set(), []
+        for sh in llama3_8b_layer_shapes():
+            if (sh.M, sh.N) not in seen:
+                seen.add((sh.M, sh.N)); shapes.append(sh)
+        batches, cfg = [1, 2, 4, 8, 16], 3
+    else:
+        shapes, cfg = llama_70b_layer_shapes(), 4
+        batches = [512] if args.workload == "gemm70b" else [1]
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    tc_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    stream = torch.cuda.Stream(device)
+    cases = []
+    sampler = ClockSampler(0)
+    t_start = time.time()
+    for sh in shapes:
+        per_layer = layer_bytes(sh.M, sh.N, 1)
+        copies = max(2, min(args.copies, int(4 * 126e6 / per_layer) + 1))
+        layers = []
+        for c in range(copies):
+            L = make_layer(sh.M, sh.N, K_PATHS, key=(cfg, c, sh.M, sh.N))
+            layers.append(rabit.rabit_pack(L.planes, L.g, L.h, device=device))
+        for batch in batches:
+            x = torch.from_numpy(make_x(batch, sh.N, key=(cfg, 10_000, batch))).to(device)
+            y = torch.zeros((batch, sh.M), dtype=torch.float16, device=device)
+            with torch.cuda.stream(stream):
+                for L in layers:
+                    rabit.rabit_linear(L, x, y)
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for L in layers:
+                    rabit.rabit_linear(L, x, y)
+            reps = max(3, args.steps // copies) if args.steps < 32000 else max(3, int(0.3 / (copies * 30e-6)))
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    g.replay()
+                ev0.record(stream)
+                for _ in range(reps):
+                    g.replay()
+                ev1.record(stream)
+            stream.synchronize()
+            us = ev0.elapsed_time(ev1) * 1e3 / (reps * copies)
+            nbytes = layer_bytes(sh.M, sh.N, batch)
+            flops = 2.0 * batch * sh.M * sh.N * K_PATHS
+            case = {"M": sh.M, "N": sh.N, "batch": batch, "copies": copies, "us_per_layer": us,
+                    "gbs": nbytes / us / 1e3, "tflops": flops / us / 1e6}
+            if batch > 16:
+                case["roofline"] = {"bound": "tensor", "achieved": case["tflops"], "peak": tc_peak, "unit": "TFLOP/s",
+                                    "frac": case["tflops"] / tc_peak}
+            else:
+                case["roofline"] = {"bound": "hbm", "achieved": case["gbs"], "peak": hbm_peak, "unit": "GB/s",
+                                    "frac": case["gbs"] / hbm_peak}
+            cases.append(case)
+            del g
+        for L in layers:
+            L.free()
+        del layers
+        torch.cuda.empty_cache()
+    clocks = sampler.summary(t_start, time.time())
+    sampler.stop()
+    head = max(cases, key=lambda c: c["M"] * c["N"] * c["batch"])
+    gemm = args.workload == "gemm70b"
+    return {"metric": "batch-512 residual-binary GEMM TFLOP/s" if gemm else METRIC,
+            "value": head["tflops"] if gemm else head["us_per_layer"], "unit": "TFLOP/s" if gemm else UNIT,
+            "n_gpus": 1, "steps": args.steps, "warmup": 3, "ms_per_step": head["us_per_layer"] / 1e3,
+            "higher_is_better": gemm, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16 tensor-core products, fp32 accumulate" if gemm else "int8 tensor-core products of exact fixed-point activations",
+            "data": "synthetic", "config": {"workload": args.workload, "K": K_PATHS,
+                                            "l2": "rotation over distinct copies of each layer, > 4 x L2 in total where the layer is small"},
+            "cases": cases, "roofline": head["roofline"], "clocks": clocks,
+            "gpu_launches": sum(c["copies"] for c in cases)}
+
+
 def bench_reference(args) -> dict:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -342,10 +430,17 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2000)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemv70b", "sweep8b"],
+                    help="decoder7b is the contract's line; the others are extra single-GPU measurements")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    res = bench_reference(args) if args.impl == "reference" else bench_rabit(args)
+    if args.impl == "reference":
+        res = bench_reference(args)
+    elif args.workload != "decoder7b":
+        res = bench_cases(args)
+    else:
+        res = bench_rabit(args)
     if res is not None:
         print(json.dumps(res))
 

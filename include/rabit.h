@@ -134,8 +134,8 @@ RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, vo
  *   - Calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on a
  *     device looks up the device address of the array (cudaGetSymbolAddress); make that first
  *     call before any stream capture begins.
- *   - All calls, for all layers, share the one array.  Each call clears the part that must start
- *     at zero (a memset enqueued on `stream` ahead of the kernel).  Two calls that overlap on the
+ *   - All calls, for all layers, share the one array.  Each call first puts the part of it that this
+ *     layer uses back into its resting state (memsets enqueued on `stream` ahead of the kernel).  Two calls that overlap on the
  *     GPU (different streams, or one stream per thread) race on it and give wrong results: keep
  *     all uses of this entry point on one stream, or serialise them yourself.
  * Results equal those of rabit_linear (same kernel, same summation order).

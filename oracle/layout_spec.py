@@ -6,7 +6,8 @@ library image can be compared byte for byte.  The paper fixes only the sign -> b
 
 Image = header (256 B) | sign tiles | g fp16 [K][Mp] | h fp16 [K][N] | fp32 partial scratch
 [n_rt*K + max_grid][partial_batch][128] | u32 flags [n_rt*K + max_grid] + one status word; every
-section starts on a 256-byte boundary; padding, scratch, flags and status are zero.
+section starts on a 256-byte boundary; padding, flags (reserved) and status are zero, the partial
+scratch section is filled with 0xFF bytes (its resting state: "nothing written yet").
 Mp = M rounded up to 128; padded signs are +1 (bit 0), padded scales 0; N is a multiple of
 32 and is not padded.  The header also records max_j |h_k[j]| per path as an fp32 bit
 pattern (the kernels derive their fixed-point scale from it).
@@ -100,6 +101,7 @@ def pack_spec(planes: np.ndarray, g: np.ndarray, h: np.ndarray) -> np.ndarray:
     tiles = np.stack([_tiles_of_plane(planes[k], M, N, geo["Mp"]) for k in range(K)], axis=1)   # [rt][k][ct][512]
     flat = tiles.reshape(-1)
     img[geo["off_bits"]:geo["off_bits"] + flat.size] = flat
+    img[geo["off_partial"]:geo["off_flags"]] = 0xFF
     gp = np.zeros((K, geo["Mp"]), dtype=np.uint16); gp[:, :M] = g16.view(np.uint16)
     img[geo["off_g"]:geo["off_g"] + gp.nbytes] = gp.view(np.uint8).reshape(-1)
     hp = np.ascontiguousarray(h16.view(np.uint16))

@@ -27,11 +27,13 @@
 //   * Eight MMA warps take the tiles of a stage round-robin: one 128-bit shared-memory read
 //     of weights, one 64-bit read of digits, 32 ANDs and 8 MMAs per 4096 weights.
 //   * A segment is the part of the CTA range inside one (row tile, path) strip.  At a
-//     segment end the warps are summed in shared memory, scaled by g_k / sigma, written to
-//     a per-layer fp32 partial buffer and published with a release store of a flag.  The
-//     CTA that owns the last tile of a row tile finishes it: it acquires the flags of the
-//     other contributors (all of them CTAs with a lower index, so the waits cannot form a
-//     cycle), adds the partials in a fixed order (deterministic) and stores fp16.
+//     segment end the warps are summed in shared memory, scaled by g_k / sigma and written to
+//     a per-layer fp32 partial buffer whose resting content is a sentinel bit pattern (all
+//     ones, a NaN no arithmetic here produces): the data is its own "published" flag.  The
+//     CTA that owns the last tile of a row tile finishes it: each of its threads reads the
+//     partials of its row from the other contributors (all of them CTAs with a lower index,
+//     so the waits cannot form a cycle), waiting (bounded) while it still sees the sentinel,
+//     puts the sentinel back, adds in a fixed order (deterministic) and stores fp16.
 // Every wait in the kernel is bounded; a wait that runs out sets a status word and the
 // kernel drains and returns (results are then invalid, the context stays usable).
 #include <cuda_fp16.h>
@@ -48,6 +50,7 @@ constexpr int kStageTiles = 16;
 constexpr int kRing = 8;
 constexpr int kBuildAhead = 3;                          // stages of raw x / h a builder lane keeps in flight
 constexpr long long kWaitLimitCycles = 1LL << 31;       // about one second
+constexpr unsigned int kSentinel = 0xFFFFFFFFu;         // resting content of the partial buffer ("not written yet")
 
 // Division of a 31-bit dividend by a constant known at launch: n / d = (umulhi(n, mul) + n) >> shr.
 struct FastDiv {
@@ -73,7 +76,7 @@ struct GemvParams {
     const __half* x;
     __half* y;
     float* partial;          // [n_rt*K + grid][RABIT_PARTIAL_BATCH][128]
-    unsigned int* flags;     // [n_rt*K + grid]: segment (CTA c, strip s) publishes its partial under index c + s
+                             // segment (CTA c, strip s) uses slot c + s; every word rests at kSentinel between calls
     unsigned int* status;
     int n_tiles;             // n_rt * K * n_ct (< 2^31)
     int q, r;                // n_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
@@ -364,10 +367,13 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     for (int b = 0; b < NB; ++b) sum_t[b] = 0;
     const int me = blockIdx.x;
     const int KC = G.K * C;
+    bool red_in_use = false;
 
-    // Segment end: sum the eight warps in shared memory, scale by g_k / sigma, store the partial row
-    // sums and publish them (unless this CTA is the one that will finish the row tile itself).
+    // Segment end: sum the eight warps in shared memory, scale by g_k / sigma and store the partial
+    // row sums; a stored word is visible to the finisher as soon as it differs from the sentinel.
     auto segment_flush = [&]() {
+        if (red_in_use) bar_mma_warps();                                       // readers of the previous flush are done
+        red_in_use = true;
         float st_f[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) {                                         // the four quarters live in lanes tq = 0..3
@@ -392,17 +398,16 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             }
         }
         bar_mma_warps();
-        const int seg_id = me + strip;
         if (reducer) {
             float sum = 0.f;
 #pragma unroll
             for (int ww = 0; ww < kMmaWarps; ++ww) sum += S.red[ww][red_b][red_r];
             const float inv = k == 0 ? sig_inv[0] : (k == 1 ? sig_inv[1] : sig_inv[2]);
-            P.partial[((size_t)seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r] = gval * (sum * inv);
+            unsigned int bits = __float_as_uint(gval * (sum * inv));
+            if (bits == kSentinel) bits = 0x7FFFFFFFu;                          // a NaN result must not look unwritten
+            const size_t seg_id = (size_t)me + strip;
+            __stcg(reinterpret_cast<unsigned int*>(P.partial) + (seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r, bits);
         }
-        bar_mma_warps();                                                        // partial stores ordered before the release; S.red free again
-        if (tid == 0 && cta_of((rt + 1) * KC - 1, P) != me)
-            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(P.flags + seg_id), "r"(1u) : "memory");
     };
 
     auto next_segment = [&]() {
@@ -474,66 +479,51 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         next_segment();
     }
 
-    // ---- finish the row tiles whose last tile this CTA owns: wait (bounded) for the flags of the other
-    //      contributors, add all partials in a fixed order, store fp16, clear the flags for the next call
-    for (int rt_f = fdiv(lo, P.div_kc); (rt_f + 1) * KC - 1 < lo + n_tiles; ++rt_f) {
-        // contributors: for every path kk the CTAs c0..c1 whose range meets strip (rt_f, kk)
-        int c0k[RABIT_MAX_K], cntk[RABIT_MAX_K];
-        int total = 0;
-        bool small = true;
-#pragma unroll
-        for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
-            c0k[kk] = 0; cntk[kk] = 0;
-            if (kk < G.K) {
-                const int s0 = (rt_f * G.K + kk) * C;
-                c0k[kk] = cta_of(s0, P);
-                cntk[kk] = cta_of(s0 + C - 1, P) - c0k[kk] + 1;
-                total += cntk[kk];
-                small = small && cntk[kk] <= 8;
-            }
-        }
-        for (int e = tid; e < total; e += kMmaThreads) {
-            int kk = 0, c = e;
-            while (c >= cntk[kk]) { c -= cntk[kk]; ++kk; }
-            c += c0k[kk];
-            if (c == me) continue;
-            const unsigned int* f = P.flags + (c + rt_f * G.K + kk);
-            unsigned int v;
-            const long long t0 = clock64();
-            while (true) {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
-                if (v) break;
-                if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
-            }
-            *const_cast<unsigned int*>(f) = 0u;                                   // leave the scratch clean for the next call
-        }
-        bar_mma_warps();
-        if (reducer) {
-            constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
-            const float* src[RABIT_MAX_K];
-#pragma unroll
-            for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-                src[kk] = P.partial + (((size_t)c0k[kk] + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+    // ---- finish the row tiles whose last tile this CTA owns.  Every reducer thread works alone on its
+    //      (batch row, row): it reads that word of every contributor's partial, path by path and CTA by
+    //      CTA, waits (bounded) while a word still holds the sentinel, restores the sentinel for the next
+    //      call, adds in that fixed order and stores fp16.  No barrier and no fence is involved: a
+    //      partial word carries no other data with it.
+    if (reducer) {
+        constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+        for (int rt_f = fdiv(lo, P.div_kc); (rt_f + 1) * KC - 1 < lo + n_tiles; ++rt_f) {
             float sum = 0.f;
-            if (small) {
-                float v[RABIT_MAX_K][8];
+#pragma unroll 1
+            for (int kk = 0; kk < G.K; ++kk) {
+                const int s0 = (rt_f * G.K + kk) * C;
+                const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
+                unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
+                                    (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+#pragma unroll 1
+                for (int c = c0; c <= c1; c += 8) {                            // eight loads in flight, consumed in order
+                    unsigned int v[8];
 #pragma unroll
-                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                    for (int u = 0; u < 8; ++u) {
+                        v[u] = 0u;
+                        if (c + u <= c1) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
+                    }
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) v[kk][u] = u < cntk[kk] ? __ldcg(src[kk] + u * kStride) : 0.f;
-#pragma unroll
-                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) sum += v[kk][u];
-            } else {
-#pragma unroll
-                for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-                    for (int c = 0; c < cntk[kk]; ++c) sum += __ldcg(src[kk] + c * kStride);
+                    for (int u = 0; u < 8; ++u) {
+                        if (c + u > c1) break;
+                        if (v[u] == kSentinel) {
+                            const long long t0 = clock64();
+                            do {
+                                asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
+                                if (v[u] != kSentinel) break;
+                                if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
+                            } while (true);
+                        }
+                        __stcg(src + u * kStride, kSentinel);
+                        sum += __uint_as_float(v[u]);
+                    }
+                    src += 8 * kStride;
+                }
             }
             const int row = rt_f * RABIT_TILE_ROWS + red_r;
             if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
         }
     }
+    bar_mma_warps();                                                           // abort_flag of every warp is final
     if (*abort_flag && tid == 0) atomicExch(P.status, 1u);
 }
 
@@ -575,7 +565,6 @@ cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, 
     P.x = (const __half*)x;
     P.y = (__half*)y;
     P.partial = L.d_partial;
-    P.flags = L.d_flags;
     P.status = L.d_status;
     P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
     int grid = 2 * (L.sm_count > 0 ? L.sm_count : 148);      // two co-resident CTAs per SM

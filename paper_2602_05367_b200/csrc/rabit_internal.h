@@ -19,8 +19,8 @@ struct rabit_layer {
     const uint4* d_bits;         // sign tiles
     const uint16_t* d_g;         // fp16 [K][Mp]
     const uint16_t* d_h;         // fp16 [K][N]
-    float* d_partial;            // fp32 [n_rt*K + RABIT_MAX_GRID][RABIT_PARTIAL_BATCH][128] cross-CTA partial sums
-    unsigned int* d_flags;       // u32 [n_rt*K + RABIT_MAX_GRID] "partial published" flags (zero between calls), then one status word
+    float* d_partial;            // fp32 [n_rt*K + RABIT_MAX_GRID][RABIT_PARTIAL_BATCH][128] cross-CTA partial sums (all-ones words between calls)
+    unsigned int* d_flags;       // u32 [n_rt*K + RABIT_MAX_GRID] reserved (zero), then one status word
     unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
 };
 

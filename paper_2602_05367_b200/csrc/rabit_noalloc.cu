@@ -2,7 +2,7 @@
 // that belongs to the library, for callers that must not allocate device memory.
 //
 // The GEMV needs two pieces of scratch per call: the fp32 partial sums that the CTAs of a row
-// tile exchange and the "partial published" flags.  rabit_linear keeps them inside the packed
+// tile exchange and a status word.  rabit_linear keeps them inside the packed
 // image that the caller allocated.  Here they live in a file-scope device array of a fixed size,
 // so the call neither needs a scratch-bearing buffer nor allocates one.
 #include <cuda_fp16.h>
@@ -14,7 +14,7 @@ namespace {
 constexpr size_t kScratchBytes = (size_t)4 << 20;        // 4 MiB, held by every GPU that loads the library
 constexpr int kMaxDevices = 64;
 
-// Partial sums | flags | status word.  Every call shares this array.
+// Partial sums | reserved | status word.  Every call shares this array.
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 // Device address of the array per device, resolved on the first call on that device.
@@ -74,7 +74,9 @@ extern "C" int rabit_linear_static_scratch(const rabit_layer* layer, const void*
     }
     unsigned char* base = g_scratch_ptr[dev];
     cudaStream_t st = (cudaStream_t)stream;
-    // The array keeps whatever the last call (of any layer) left: flags and status must start at zero.
+    // The array keeps whatever the last call (of any layer) left: the partial slots of this layer must
+    // start in their resting state (all-ones words) and the status word at zero.
+    RABIT_CUDA_TRY(cudaMemsetAsync(base, 0xFF, plan.partial_bytes, st));
     RABIT_CUDA_TRY(cudaMemsetAsync(base + plan.flags_off, 0, plan.status_off + 256 - plan.flags_off, st));
 
     rabit_layer view = *layer;                               // same weights and scales, scratch redirected

@@ -126,6 +126,7 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
     uint8_t* base = (uint8_t*)out;
     std::memset(base, 0, hdr.total_bytes);
     std::memcpy(base, &hdr, sizeof(hdr));
+    std::memset(base + hdr.off_partial, 0xFF, hdr.off_flags - hdr.off_partial);   // resting state of the partial buffer
 
     uint8_t* bits = base + hdr.off_bits;
     const size_t plane_words = (size_t)M * (N / 32);

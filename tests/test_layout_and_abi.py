@@ -88,7 +88,8 @@ def test_scratch_and_padding_are_zero():
     L = make_layer(40, 160, 2, key=(84,))
     img = rabit.pack_host(L.planes, L.g, L.h)
     hd = spec.read_header(img)
-    assert not img[hd["off_partial"]:hd["total_bytes"]].any()
+    assert (img[hd["off_partial"]:hd["off_flags"]] == 0xFF).all()       # resting state of the partial buffer
+    assert not img[hd["off_flags"]:hd["total_bytes"]].any()
     g = img[hd["off_g"]:hd["off_h"]].view(np.uint16)[:2 * hd["Mp"]].reshape(2, hd["Mp"])
     assert not g[:, 40:].any()
 
