@@ -48,6 +48,7 @@ constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kThreads = (kMmaWarps + kBuildWarps) * 32;
 constexpr int kStageTiles = 16;
 constexpr int kRing = 8;
+constexpr int kHeadStages = kMmaWarps / kBuildWarps;    // first stages, built by the (still idle) MMA warps, one warp pair each
 constexpr int kBuildAhead = 3;                          // stages of raw x / h a builder lane keeps in flight
 constexpr long long kWaitLimitCycles = 1LL << 31;       // about one second
 constexpr unsigned int kSentinel = 0xFFFFFFFFu;         // resting content of the partial buffer ("not written yet")
@@ -193,15 +194,18 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     }
     // Builder lanes: lane index bi = 0..63 of the two builder warps takes tile bi >> 2 of every stage
     // and columns 8*(bi & 3) .. +7 of it.
-    const int bw = warp - kMmaWarps;
-    const int bi = ((bw & 1) << 5) | lane;
+    // The first kHeadStages stages are built by the MMA warps (pair warp >> 1 takes stage warp >> 1),
+    // which have nothing else to do until a table exists; the builder warps start behind them.
+    const int bi = ((warp & 1) << 5) | lane;
     const int bj = bi >> 2, bv = bi & 3;
-    int pf_ct = 0, pf_k = 0, pf_stage = 0;           // (column tile, path, stage) of the next prefetch
+    int pf_ct = 0, pf_k = 0;                          // (column tile, path) of the next prefetch / of the head stage
+    int pf_stage = warp >= kMmaWarps ? kHeadStages : (warp >> 1);
     uint4 hq[kBuildAhead];
-    if (warp >= kMmaWarps) {
-        const int p0 = lo + bj;
-        pf_ct = fmod(p0, P.div_c);
-        pf_k = fmod(fdiv(p0, P.div_c), P.div_k);
+    {
+        const int p0 = lo + pf_stage * kStageTiles + bj;
+        const int st0 = fdiv(p0, P.div_c);
+        pf_ct = p0 - st0 * C;
+        pf_k = fmod(st0, P.div_k);
     }
     auto prefetch_h = [&](int d) {                   // input scales: static data, may be read before the wait
         hq[d] = make_uint4(0u, 0u, 0u, 0u);
@@ -216,13 +220,20 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     const int red_b = (tid >> 7) & 1, red_r = tid & 127;                   // (batch row, row) this thread reduces
     const bool reducer = warp < kMmaWarps && red_b < NB;
     float gval = 0.f;
-    if (warp >= kMmaWarps) {
-        if (kBuildAhead > 0) prefetch_h(0);
-    } else if (reducer && n_tiles > 0) {
-        gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
-    }
+    prefetch_h(0);                                   // builder: its first stage; MMA warp: its head stage
+    if (reducer && n_tiles > 0) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 
     asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    uint4 head_x[NB];                                // MMA warps: activations of the head stage, in flight during the max pass
+#pragma unroll
+    for (int b = 0; b < NB; ++b) head_x[b] = make_uint4(0u, 0u, 0u, 0u);
+    const bool head_live = warp < kMmaWarps && pf_stage < n_stages && pf_stage * kStageTiles + bj < n_tiles;
+    if (head_live) {
+#pragma unroll
+        for (int b = 0; b < NB; ++b)
+            head_x[b] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
+    }
 
     // ---- largest |x| per batch row (fp16 bit patterns order like unsigned integers once the sign is cleared)
     {
@@ -245,17 +256,52 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     __syncthreads();
     if (n_tiles == 0) return;
 
+    // One lane's share of a stage: columns 8*bv .. +7 of tile j, all batch rows -> digit words + sum of T.
+    auto build_part = [&](int slot, int j, int kk, const uint4& hraw, const uint4 (&xraw)[NB], const float (&sg_b)[NB][RABIT_MAX_K]) {
+        const uint32_t hw[4] = {hraw.x, hraw.y, hraw.z, hraw.w};
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const float sg = kk == 0 ? sg_b[b][0] : (kk == 1 ? sg_b[b][1] : sg_b[b][2]);
+            const uint32_t xw[4] = {xraw[b].x, xraw[b].y, xraw[b].z, xraw[b].w};
+            int Tq[8];
+#pragma unroll
+            for (int c2 = 0; c2 < 4; ++c2) {
+                const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[c2]));
+                const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[c2]));
+                Tq[2 * c2] = __float2int_rn(hf.x * xf.x * sg);
+                Tq[2 * c2 + 1] = __float2int_rn(hf.y * xf.y * sg);
+            }
+            int tsum = 0;                        // |T| < 2^28, so eight of them fit
+#pragma unroll
+            for (int c = 0; c < 8; ++c) tsum += Tq[c];
+            uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][b * 16]);
+#pragma unroll
+            for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
+                const int u = 2 * bv + hlf;
+                uint32_t X[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
+                const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
+                const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
+                uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
+                dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
+                dst[8] = __byte_perm(t0, t1, 0x7632);
+                dst[16] = __byte_perm(t2, t3, 0x5410);
+                dst[24] = __byte_perm(t2, t3, 0x7632);
+            }
+            S.sum_t[slot][j][b][bv] = tsum;
+        }
+    };
+    float sigma[NB][RABIT_MAX_K], sigma_inv[NB][RABIT_MAX_K];
+#pragma unroll
+    for (int b = 0; b < NB; ++b)
+#pragma unroll
+        for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+            choose_scale(S.xmax_bits[b], kk < G.K ? G.hmax[kk] : 0.f, sigma[b][kk], sigma_inv[b][kk]);
+
     if (warp >= kMmaWarps) {
         // =========================== builder warps (and the copy issuers) ===========================
         const int j = bj;
-        float sigma[NB][RABIT_MAX_K];
-#pragma unroll
-        for (int b = 0; b < NB; ++b)
-#pragma unroll
-            for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
-                float inv;
-                choose_scale(S.xmax_bits[b], kk < G.K ? G.hmax[kk] : 0.f, sigma[b][kk], inv);
-            }
         // a queue of kBuildAhead of this pair's stages of raw inputs hides the load latency
         uint4 xq[kBuildAhead][NB];
         int kq[kBuildAhead];
@@ -273,13 +319,13 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             while (pf_ct >= C) { pf_ct -= C; pf_k = pf_k + 1 == G.K ? 0 : pf_k + 1; }
         };
 #pragma unroll
-        for (int d = 0; d < kBuildAhead; ++d) {          // stage 0's h part was fetched before the wait
+        for (int d = 0; d < kBuildAhead; ++d) {          // the first stage's h part was fetched before the wait
             if (d > 0) prefetch_h(d);
             prefetch_x(d);
         }
 
         const bool issuer = tid == kMmaThreads;          // one lane issues the copies
-        for (int i0 = 0; i0 < n_stages; i0 += kBuildAhead) {
+        for (int i0 = kHeadStages; i0 < n_stages; i0 += kBuildAhead) {
 #pragma unroll
             for (int d = 0; d < kBuildAhead; ++d) {
                 const int i = i0 + d;
@@ -295,40 +341,7 @@ rabit_gemv_mma_kernel(const GemvParams P) {
                                  tiles * RABIT_TILE_BYTES, bar);
                     }
                 }
-                const int kk = kq[d];
-                const uint32_t hw[4] = {hq[d].x, hq[d].y, hq[d].z, hq[d].w};
-#pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    const float sg = kk == 0 ? sigma[b][0] : (kk == 1 ? sigma[b][1] : sigma[b][2]);
-                    const uint32_t xw[4] = {xq[d][b].x, xq[d][b].y, xq[d][b].z, xq[d][b].w};
-                    int Tq[8];
-#pragma unroll
-                    for (int c2 = 0; c2 < 4; ++c2) {
-                        const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[c2]));
-                        const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[c2]));
-                        Tq[2 * c2] = __float2int_rn(hf.x * xf.x * sg);
-                        Tq[2 * c2 + 1] = __float2int_rn(hf.y * xf.y * sg);
-                    }
-                    int tsum = 0;                        // |T| < 2^28, so eight of them fit
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) tsum += Tq[c];
-                    uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][b * 16]);
-#pragma unroll
-                    for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
-                        const int u = 2 * bv + hlf;
-                        uint32_t X[4];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
-                        const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
-                        const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
-                        uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
-                        dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
-                        dst[8] = __byte_perm(t0, t1, 0x7632);
-                        dst[16] = __byte_perm(t2, t3, 0x5410);
-                        dst[24] = __byte_perm(t2, t3, 0x7632);
-                    }
-                    S.sum_t[slot][j][b][bv] = tsum;
-                }
+                build_part(slot, j, kq[d], hq[d], xq[d], sigma);
                 prefetch_h(d);
                 prefetch_x(d);
                 __syncwarp();
@@ -350,12 +363,14 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     // ======================================= MMA warps =======================================
     const int gq = lane >> 2, tq = lane & 3;
     const int w = warp;
+    if (pf_stage < n_stages) {                // head stage of this warp pair (slot = stage: the ring is not yet reused)
+        if (head_live) build_part(pf_stage, bj, pf_k, hq[0], head_x, sigma);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&S.full[pf_stage]));
+    }
     float sig_inv[RABIT_MAX_K];               // 1 / sigma of this thread's batch row at reduction time
 #pragma unroll
-    for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
-        float sg;
-        choose_scale(S.xmax_bits[red_b < NB ? red_b : 0], kk < G.K ? G.hmax[kk] : 0.f, sg, sig_inv[kk]);
-    }
+    for (int kk = 0; kk < RABIT_MAX_K; ++kk) sig_inv[kk] = red_b < NB ? sigma_inv[red_b < NB ? red_b : 0][kk] : 1.f;
 
     int acc[8][4];
     long long sum_t[NB];
