@@ -101,6 +101,21 @@ RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16
 RABIT_API int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
 /*
+ * Several layers that do not depend on one another in ONE launch (the same operation as rabit_linear,
+ * Section 4.1 forward with the Eq. 2 weight, per layer): layer l maps xs[l] ([batch][N_l]) to ys[l]
+ * ([batch][M_l]).  Meant for projections that read the same activations (q|k|v, gate|up: pass the same
+ * pointer several times in xs) - at batch 1 a layer lasts a few microseconds, and the fixed cost of a
+ * launch (dependency wait, first memory round trips, cross-CTA reduction) is paid once per group instead
+ * of once per layer.  The tiles of all layers are split evenly over the CTAs as if they were one layer.
+ *   layers, xs, ys   HOST arrays of n_layers entries (1 <= n_layers <= 8); the pointers inside are as for
+ *                    rabit_linear; outputs must not overlap one another nor any input; all layers on one device.
+ * For batch > 16, or more than 8 layers, the layers are simply run one after the other.
+ * Asynchronous on `stream`, allocates nothing, may be captured in a CUDA graph.
+ */
+RABIT_API int rabit_linear_group(const rabit_layer* const* layers, const void* const* xs, void* const* ys,
+                       int n_layers, int batch, void* stream);
+
+/*
  * Host-buffer form of rabit_linear (same operation, Section 4.1 forward with the Eq. 2 weight)
  * for callers whose activations live in host memory:
  *   x_host  HOST fp16 [batch][N]   (pinned memory makes the copies asynchronous)

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     unpack_host,
     rabit_pack,
     rabit_linear,
+    rabit_linear_group,
     rabit_linear_host,
     rabit_linear_static_scratch,
     rabit_free,

@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     lib.rabit_stage_bytes.argtypes = [_c_void_p, _c_int]
     lib.rabit_linear_host.restype = _c_int
     lib.rabit_linear_host.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]
+    lib.rabit_linear_group.restype = _c_int
+    lib.rabit_linear_group.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]
     lib.rabit_linear_static_scratch.restype = _c_int
     lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
     lib.rabit_unpack.restype = _c_int
@@ -196,6 +198,28 @@ def rabit_linear(layer: RabitLayer, x, y=None, stream: Optional[int] = None):
     st = torch.cuda.current_stream(x.device).cuda_stream if stream is None else stream
     _check(_lib.rabit_linear(layer.handle, _c_void_p(xb.data_ptr()), _c_void_p(y.data_ptr()), batch, _c_void_p(st)))
     return y if x.dim() == 2 else y.view(-1)
+
+
+def rabit_linear_group(layers, xs, ys, stream: Optional[int] = None):
+    """Independent layers in one launch: ys[l] = layers[l](xs[l]).  xs may repeat one tensor (projections
+    that share their input).  All tensors are contiguous CUDA float16, [batch][N_l] and [batch][M_l]."""
+    import torch
+
+    n = len(layers)
+    if n < 1 or len(xs) != n or len(ys) != n:
+        raise ValueError("layers, xs and ys must have the same, non-zero length")
+    batch = 1 if xs[0].dim() == 1 else xs[0].shape[0]
+    for L, x, y in zip(layers, xs, ys):
+        if x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous() or x.numel() != batch * L.N:
+            raise ValueError("every x must be a contiguous CUDA float16 tensor of batch*N elements")
+        if y.dtype != torch.float16 or not y.is_cuda or not y.is_contiguous() or y.numel() != batch * L.M:
+            raise ValueError("every y must be a contiguous CUDA float16 tensor of batch*M elements")
+    st = torch.cuda.current_stream(xs[0].device).cuda_stream if stream is None else stream
+    h = (_c_void_p * n)(*[L.handle for L in layers])
+    xp = (_c_void_p * n)(*[x.data_ptr() for x in xs])
+    yp = (_c_void_p * n)(*[y.data_ptr() for y in ys])
+    _check(_lib.rabit_linear_group(h, xp, yp, n, batch, _c_void_p(st)))
+    return ys
 
 
 def rabit_linear_host(layer: RabitLayer, x_host, y_host, stream: Optional[int] = None):

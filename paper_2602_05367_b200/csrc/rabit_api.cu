@@ -124,6 +124,52 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
     return RABIT_OK;
 }
 
+extern "C" int rabit_linear_group(const rabit_layer* const* layers, const void* const* xs, void* const* ys,
+                                  int n_layers, int batch, void* stream) {
+    rabit_clear_error();
+    if (!layers || !xs || !ys) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: null array");
+    if (n_layers < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: n_layers must be >= 1 (got %d)", n_layers);
+    if (batch < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: batch must be >= 1 (got %d)", batch);
+    for (int l = 0; l < n_layers; ++l) {
+        if (!layers[l] || !xs[l] || !ys[l]) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: null entry %d", l);
+        if ((((uintptr_t)xs[l]) & 15u) || (((uintptr_t)ys[l]) & 15u))
+            return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: x and y of entry %d must be 16-byte aligned", l);
+        if (layers[l]->device != layers[0]->device)
+            return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: entry %d lives on another device", l);
+    }
+    for (int a = 0; a < n_layers; ++a) {
+        const size_t ya = (size_t)batch * layers[a]->geom.M * 2;
+        for (int b = 0; b < n_layers; ++b) {
+            if (ranges_overlap(ys[a], ya, xs[b], (size_t)batch * layers[b]->geom.N * 2))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: output %d overlaps input %d", a, b);
+            if (b > a && ranges_overlap(ys[a], ya, ys[b], (size_t)batch * layers[b]->geom.M * 2))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: outputs %d and %d overlap", a, b);
+        }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    bool fused = rabit_gemv_mma_group_supports(layers, n_layers, batch);
+    for (int l = 0; l < n_layers && fused; ++l) fused = layers[l]->variant == 0 || layers[l]->variant == 2;
+    if (!fused) {
+        for (int l = 0; l < n_layers; ++l) {
+            int rc = rabit_linear(layers[l], xs[l], ys[l], batch, stream);
+            if (rc != RABIT_OK) return rc;
+        }
+        return RABIT_OK;
+    }
+    const void* xb[8];
+    void* yb[8];
+    cudaError_t e = cudaSuccess;
+    for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += 2) {            // two batch rows share one pass over the weights
+        for (int l = 0; l < n_layers; ++l) {
+            xb[l] = (const char*)xs[l] + (size_t)b0 * layers[l]->geom.N * 2;
+            yb[l] = (char*)ys[l] + (size_t)b0 * layers[l]->geom.M * 2;
+        }
+        e = rabit_launch_gemv_mma_group(layers, n_layers, xb, yb, batch - b0 >= 2 ? 2 : 1, st);
+    }
+    if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear_group: launch failed: %s", cudaGetErrorString(e));
+    return RABIT_OK;
+}
+
 extern "C" size_t rabit_stage_bytes(const rabit_layer* layer, int batch) {
     if (!layer || batch < 1) return 0;
     return rabit_align256((size_t)batch * layer->geom.N * 2) + rabit_align256((size_t)batch * layer->geom.M * 2);

@@ -78,10 +78,22 @@ struct GemvParams {
     __half* y;
     float* partial;          // [n_rt*K + grid][RABIT_PARTIAL_BATCH][128]
                              // segment (CTA c, strip s) uses slot c + s; every word rests at kSentinel between calls
+    int n_tiles;             // n_rt * K * n_ct
+    int base;                // position of this layer's first tile in the launch's tile numbering
+    FastDiv div_c, div_k, div_kc;   // by n_ct, K, K * n_ct
+};
+
+// A launch runs up to kMaxGroup layers that do not depend on one another (for example the
+// projections that read the same activations); their tiles are numbered one layer after the
+// other and that whole range is split evenly over the CTAs.
+constexpr int kMaxGroup = 8;
+struct GroupParams {
+    int n_layers;
+    int total_tiles;         // < 2^31
+    int q, r;                // total_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
+    FastDiv div_q, div_q1;   // by q, q + 1
     unsigned int* status;
-    int n_tiles;             // n_rt * K * n_ct (< 2^31)
-    int q, r;                // n_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
-    FastDiv div_c, div_k, div_kc, div_q, div_q1;   // by n_ct, K, K * n_ct, q, q + 1
+    GemvParams layer[kMaxGroup];
 };
 
 template <int NB>
@@ -134,9 +146,9 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 
 // Even split of the tile positions: CTA c owns [c*q + min(c, r), (c+1)*q + min(c+1, r)).
 __device__ __forceinline__ int range_lo(int c, int q, int r) { return c * q + min(c, r); }
-__device__ __forceinline__ int cta_of(int p, const GemvParams& P) {
-    const int big = P.r * (P.q + 1);             // positions owned by the CTAs that have q+1 tiles
-    return p < big ? fdiv(p, P.div_q1) : P.r + fdiv(p - big, P.div_q);
+__device__ __forceinline__ int cta_of(int p, const GroupParams& GP) {
+    const int big = GP.r * (GP.q + 1);           // positions owned by the CTAs that have q+1 tiles
+    return p < big ? fdiv(p, GP.div_q1) : GP.r + fdiv(p - big, GP.div_q);
 }
 
 // sigma = 2^s with |h x| * sigma < 2^28 for every column; inv = 2^-s (NaN if the inputs are not finite).
@@ -157,15 +169,12 @@ __device__ __forceinline__ void choose_scale(unsigned int xmax_bits, float hmax,
 
 template <int NB>
 __global__ void __launch_bounds__(kThreads, 2)
-rabit_gemv_mma_kernel(const GemvParams P) {
+rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem<NB>& S = *reinterpret_cast<Smem<NB>*>(smem_raw);
-    const RabitGeom& G = P.G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int C = G.n_ct;
-    const int lo = range_lo(blockIdx.x, P.q, P.r);
-    const int n_tiles = range_lo(blockIdx.x + 1, P.q, P.r) - lo;
-    const int n_stages = (n_tiles + kStageTiles - 1) / kStageTiles;
+    const int glo = range_lo(blockIdx.x, GP.q, GP.r);                      // this CTA's range in the launch's numbering
+    const int ghi = range_lo(blockIdx.x + 1, GP.q, GP.r);
     volatile int* abort_flag = &S.abort_flag;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -180,15 +189,35 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     }
     __syncthreads();
 
+    // One pass per layer that meets this CTA's range.  `it0` counts the stages of the earlier passes: the
+    // ring slots and barrier phases simply continue from pass to pass.
+    int it0 = 0;
+    bool first_pass = true;
+    for (int li = 0; li < GP.n_layers; ++li) {
+    const GemvParams& P = GP.layer[li];
+    if (P.base + P.n_tiles <= glo || P.base >= ghi) continue;
+    const RabitGeom& G = P.G;
+    const int C = G.n_ct;
+    const int lo = max(glo, P.base) - P.base;                              // this pass's range, in the layer's own numbering
+    const int n_tiles = min(ghi, P.base + P.n_tiles) - P.base - lo;
+    const int n_stages = (n_tiles + kStageTiles - 1) / kStageTiles;
+    if (!first_pass) {                                                     // every warp is done with the previous pass
+        __syncthreads();
+        if (tid < NB) S.xmax_bits[tid] = 0;
+        __syncthreads();
+    }
+
     // ---- everything that does not depend on the stream's past starts now: the first ring-full of
     //      weights, the first input scales of the builder lanes, the first output scales
     if (tid == kMmaThreads) {
         const int prefetched = n_stages < kRing ? n_stages : kRing;
         for (int i = 0; i < prefetched; ++i) {
+            const int it = it0 + i, slot = it % kRing;
+            if (it >= kRing) mbar_wait(smem_u32(&S.empty[slot]), ((it / kRing) - 1) & 1, abort_flag);
             const int tiles = min(kStageTiles, n_tiles - i * kStageTiles);
-            const uint32_t bar = smem_u32(&S.full[i]);
+            const uint32_t bar = smem_u32(&S.full[slot]);
             mbar_expect_tx(bar, tiles * RABIT_TILE_BYTES);
-            bulk_g2s(smem_u32(&S.bits[i][0][0]), P.bits + ((size_t)lo + (size_t)i * kStageTiles) * RABIT_TILE_BYTES,
+            bulk_g2s(smem_u32(&S.bits[slot][0][0]), P.bits + ((size_t)lo + (size_t)i * kStageTiles) * RABIT_TILE_BYTES,
                      tiles * RABIT_TILE_BYTES, bar);
         }
     }
@@ -223,7 +252,8 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     prefetch_h(0);                                   // builder: its first stage; MMA warp: its head stage
     if (reducer && n_tiles > 0) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (first_pass) asm volatile("griddepcontrol.wait;" ::: "memory");
+    first_pass = false;
 
     uint4 head_x[NB];                                // MMA warps: activations of the head stage, in flight during the max pass
 #pragma unroll
@@ -254,7 +284,6 @@ rabit_gemv_mma_kernel(const GemvParams P) {
         }
     }
     __syncthreads();
-    if (n_tiles == 0) return;
 
     // One lane's share of a stage: columns 8*bv .. +7 of tile j, all batch rows -> digit words + sum of T.
     auto build_part = [&](int slot, int j, int kk, const uint4& hraw, const uint4 (&xraw)[NB], const float (&sg_b)[NB][RABIT_MAX_K]) {
@@ -330,9 +359,9 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             for (int d = 0; d < kBuildAhead; ++d) {
                 const int i = i0 + d;
                 if (i >= n_stages) break;
-                const int slot = i % kRing;
+                const int slot = (it0 + i) % kRing;
                 if (i >= kRing) {
-                    mbar_wait(smem_u32(&S.empty[slot]), ((i / kRing) - 1) & 1, abort_flag);
+                    mbar_wait(smem_u32(&S.empty[slot]), (((it0 + i) / kRing) - 1) & 1, abort_flag);
                     if (issuer) {
                         const int tiles = min(kStageTiles, n_tiles - i * kStageTiles);
                         const uint32_t bar = smem_u32(&S.full[slot]);
@@ -348,25 +377,15 @@ rabit_gemv_mma_kernel(const GemvParams P) {
                 if (lane == 0) mbar_arrive(smem_u32(&S.full[slot]));
             }
         }
-        if (*abort_flag && issuer) {
-            // make sure no bulk copy is still in flight towards this CTA's shared memory
-            for (int i = max(0, n_stages - kRing); i < n_stages; ++i) {
-                const long long t0 = clock64();
-                while (!mbar_try_wait(smem_u32(&S.full[i % kRing]), (i / kRing) & 1))
-                    if (clock64() - t0 > kWaitLimitCycles) break;
-            }
-            atomicExch(P.status, 1u);
-        }
-        return;
-    }
-
+    } else {
     // ======================================= MMA warps =======================================
     const int gq = lane >> 2, tq = lane & 3;
     const int w = warp;
-    if (pf_stage < n_stages) {                // head stage of this warp pair (slot = stage: the ring is not yet reused)
-        if (head_live) build_part(pf_stage, bj, pf_k, hq[0], head_x, sigma);
+    if (pf_stage < n_stages) {                // head stage of this warp pair (its slot's earlier use ended with the previous pass)
+        const int hslot = (it0 + pf_stage) % kRing;
+        if (head_live) build_part(hslot, bj, pf_k, hq[0], head_x, sigma);
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.full[pf_stage]));
+        if (lane == 0) mbar_arrive(smem_u32(&S.full[hslot]));
     }
     float sig_inv[RABIT_MAX_K];               // 1 / sigma of this thread's batch row at reduction time
 #pragma unroll
@@ -456,10 +475,10 @@ rabit_gemv_mma_kernel(const GemvParams P) {
     };
 #pragma unroll 1
     for (int i = 0; i < n_stages; ++i) {
-        const int slot = i % kRing;
+        const int slot = (it0 + i) % kRing;
         const int rel0 = i * kStageTiles + w, rel1 = rel0 + kMmaWarps;
         if (rel0 >= n_tiles) break;
-        mbar_wait(smem_u32(&S.full[slot]), (i / kRing) & 1, abort_flag);
+        mbar_wait(smem_u32(&S.full[slot]), ((it0 + i) / kRing) & 1, abort_flag);
         if (rel1 < seg_end) {
             const uint4 wa = S.bits[slot][w][lane];
             const uint4 wb = S.bits[slot][w + kMmaWarps][lane];
@@ -506,7 +525,7 @@ rabit_gemv_mma_kernel(const GemvParams P) {
 #pragma unroll 1
             for (int kk = 0; kk < G.K; ++kk) {
                 const int s0 = (rt_f * G.K + kk) * C;
-                const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
+                const int c0 = cta_of(P.base + s0, GP), c1 = cta_of(P.base + s0 + C - 1, GP);
                 unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
                                     (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
 #pragma unroll 1
@@ -538,8 +557,20 @@ rabit_gemv_mma_kernel(const GemvParams P) {
             if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
         }
     }
-    bar_mma_warps();                                                           // abort_flag of every warp is final
-    if (*abort_flag && tid == 0) atomicExch(P.status, 1u);
+    }                                                                          // MMA warps
+    it0 += n_stages;
+    }                                                                          // passes
+
+    __syncthreads();                                                           // abort_flag of every warp is final
+    if (*abort_flag && tid == kMmaThreads) {
+        // make sure no bulk copy is still in flight towards this CTA's shared memory
+        for (int it = max(0, it0 - kRing); it < it0; ++it) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&S.full[it % kRing]), (it / kRing) & 1))
+                if (clock64() - t0 > kWaitLimitCycles) break;
+        }
+        atomicExch(GP.status, 1u);
+    }
 }
 
 }  // namespace
@@ -550,7 +581,7 @@ bool rabit_gemv_mma_supports(const rabit_layer& L, int batch) {
 }
 
 template <int NB>
-static cudaError_t launch_nb(const GemvParams& P, int grid, cudaStream_t stream) {
+static cudaError_t launch_nb(const GroupParams& GP, int grid, cudaStream_t stream) {
     static bool attr_done = false;
     const size_t smem = sizeof(Smem<NB>);
     if (!attr_done) {
@@ -568,29 +599,55 @@ static cudaError_t launch_nb(const GemvParams& P, int grid, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rabit_gemv_mma_kernel<NB>, P);
+    return cudaLaunchKernelEx(&cfg, rabit_gemv_mma_kernel<NB>, GP);
+}
+
+int rabit_gemv_mma_max_group() { return kMaxGroup; }
+
+bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch) {
+    if (n_layers < 1 || n_layers > kMaxGroup || batch < 1 || batch > RABIT_MAX_GEMV_BATCH) return false;
+    long long tiles = 0;
+    for (int l = 0; l < n_layers; ++l) tiles += (long long)layers[l]->geom.n_rt * layers[l]->geom.K * layers[l]->geom.n_ct;
+    return tiles < (1LL << 31);
+}
+
+// One launch for n_layers independent layers, one or two batch rows (x_l: [batch][N_l], y_l: [batch][M_l]).
+cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
+                                        int batch, cudaStream_t stream) {
+    GroupParams GP;
+    GP.n_layers = n_layers;
+    GP.total_tiles = 0;
+    GP.status = layers[0]->d_status;
+    for (int l = 0; l < n_layers; ++l) {
+        const rabit_layer& L = *layers[l];
+        GemvParams& P = GP.layer[l];
+        P.G = L.geom;
+        P.bits = reinterpret_cast<const unsigned char*>(L.d_bits);
+        P.g = (const __half*)L.d_g;
+        P.h = (const __half*)L.d_h;
+        P.x = (const __half*)xs[l];
+        P.y = (__half*)ys[l];
+        P.partial = L.d_partial;
+        P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
+        P.base = GP.total_tiles;
+        P.div_c = make_fastdiv((unsigned int)L.geom.n_ct);
+        P.div_k = make_fastdiv((unsigned int)L.geom.K);
+        P.div_kc = make_fastdiv((unsigned int)(L.geom.K * L.geom.n_ct));
+        GP.total_tiles += P.n_tiles;
+    }
+    for (int l = n_layers; l < kMaxGroup; ++l) GP.layer[l] = GP.layer[0];
+    const int sms = layers[0]->sm_count > 0 ? layers[0]->sm_count : 148;
+    int grid = 2 * sms;                                      // two co-resident CTAs per SM
+    if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
+    if (grid > GP.total_tiles) grid = GP.total_tiles;
+    GP.q = GP.total_tiles / grid;
+    GP.r = GP.total_tiles % grid;
+    GP.div_q = make_fastdiv((unsigned int)GP.q);
+    GP.div_q1 = make_fastdiv((unsigned int)GP.q + 1u);
+    return batch == 1 ? launch_nb<1>(GP, grid, stream) : launch_nb<2>(GP, grid, stream);
 }
 
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
-    GemvParams P;
-    P.G = L.geom;
-    P.bits = reinterpret_cast<const unsigned char*>(L.d_bits);
-    P.g = (const __half*)L.d_g;
-    P.h = (const __half*)L.d_h;
-    P.x = (const __half*)x;
-    P.y = (__half*)y;
-    P.partial = L.d_partial;
-    P.status = L.d_status;
-    P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
-    int grid = 2 * (L.sm_count > 0 ? L.sm_count : 148);      // two co-resident CTAs per SM
-    if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
-    if (grid > P.n_tiles) grid = P.n_tiles;
-    P.q = P.n_tiles / grid;
-    P.r = P.n_tiles % grid;
-    P.div_c = make_fastdiv((unsigned int)L.geom.n_ct);
-    P.div_k = make_fastdiv((unsigned int)L.geom.K);
-    P.div_kc = make_fastdiv((unsigned int)(L.geom.K * L.geom.n_ct));
-    P.div_q = make_fastdiv((unsigned int)P.q);
-    P.div_q1 = make_fastdiv((unsigned int)P.q + 1u);
-    return batch == 1 ? launch_nb<1>(P, grid, stream) : launch_nb<2>(P, grid, stream);
+    const rabit_layer* one = &L;
+    return rabit_launch_gemv_mma_group(&one, 1, &x, &y, batch, stream);
 }
