@@ -134,9 +134,22 @@ def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: 
     return shapes, layers, xs, xs_host, ys
 
 
-def run_step(rabit, shapes, layer_row, xs, ys, token: int):
-    for p, sh in enumerate(shapes):
-        rabit.rabit_linear(layer_row[p], xs[sh.N][token], ys[p])
+# Projections of a decoder layer that read the same activations: q|k|v and gate|up go through
+# rabit_linear_group (one launch each), o and down through rabit_linear.
+GROUPS = [[0, 1, 2], [3], [4, 5], [6]]
+
+
+def run_step(rabit, shapes, layer_row, xs, ys, token: int, grouped: bool = True):
+    if not grouped:
+        for p, sh in enumerate(shapes):
+            rabit.rabit_linear(layer_row[p], xs[sh.N][token], ys[p])
+        return
+    for grp in GROUPS:
+        if len(grp) == 1:
+            p = grp[0]
+            rabit.rabit_linear(layer_row[p], xs[shapes[p].N][token], ys[p])
+        else:
+            rabit.rabit_linear_group([layer_row[p] for p in grp], [xs[shapes[p].N][token] for p in grp], [ys[p] for p in grp])
 
 
 # ---------------------------------------------------------------------------------------
@@ -175,12 +188,14 @@ def bench_rabit(args) -> dict:
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
             for c in copy_ids:
-                run_step(rabit, shapes, layers[c], xs, ys, c % tokens)
+                run_step(rabit, shapes, layers[c], xs, ys, c % tokens, grouped)
         return g
 
+    grouped = not args.no_group
+    launches_per_step = len(GROUPS) if grouped else n_proj
     with torch.cuda.stream(stream):
         for c in range(copies):                      # also the first-call set-up of every kernel variant
-            run_step(rabit, shapes, layers[c], xs, ys, c % tokens)
+            run_step(rabit, shapes, layers[c], xs, ys, c % tokens, grouped)
     stream.synchronize()
     use_graph = not args.no_graph
     if use_graph:
@@ -193,7 +208,7 @@ def bench_rabit(args) -> dict:
         with torch.cuda.stream(stream):
             while s < end:
                 if not use_graph:
-                    run_step(rabit, shapes, layers[s % copies], xs, ys, (s % copies) % tokens)
+                    run_step(rabit, shapes, layers[s % copies], xs, ys, (s % copies) % tokens, grouped)
                     s += 1
                 elif s % copies == 0 and end - s >= copies:
                     cycle_graph.replay(); s += copies
@@ -276,10 +291,13 @@ def bench_rabit(args) -> dict:
                    "packed_bytes_total": int(step_bytes * copies),
                    "l2": "inputs larger than L2: rotation over %d distinct decoder layers (%.0f MB)" % (copies, step_bytes * copies / 1e6),
                    "launch": "CUDA graph replay" if use_graph else "stream launches",
+                   "launches_per_step": launches_per_step,
+                   "grouping": "q|k|v and gate|up (projections that share their input) each go through one rabit_linear_group launch; "
+                               "o and down through rabit_linear" if grouped else "one rabit_linear launch per projection",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "achieved_hbm_gbs": gbs * world,
         "tokens_per_s_32_layer_stack": world * 1.0 / (32 * ms_per_step * 1e-3),
-        "gpu_launches": args.steps * n_proj,
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
@@ -440,6 +458,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=2000)
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-group", action="store_true", help="one rabit_linear launch per projection (7 per step instead of 4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemv70b", "sweep8b"],
                     help="decoder7b is the contract's line; the others are extra single-GPU measurements")
