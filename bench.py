@@ -29,6 +29,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) of the four launches of one grouped step, from the ncu capture summarised in
+# profiles/gemv_mma_llama2_7b_decoder_layer.md (12.760 + 4.294 + 22.770 + 11.415 MB); valid for the
+# default grouped batch-1 workload only.
+NCU_DRAM_BYTES_PER_GROUPED_STEP = 51_239_424
+
 METRIC = "batch-1 residual-binary GEMV us/layer"
 UNIT = "us/layer"
 WORKLOAD = "llama2-7b decoder layer: 7 residual-binary projections, K=2, batch 1, back to back"
@@ -301,8 +306,11 @@ def bench_rabit(args) -> dict:
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": None, "peak_source": peak_src,
-                     "note": "algorithmic bytes of the seven layers of a step / device time of a step (launch gaps included)"},
+                     "traffic": (NCU_DRAM_BYTES_PER_GROUPED_STEP / launches_per_step) if (grouped and batch == 1) else None,
+                     "algorithmic_bytes_per_launch": step_bytes / launches_per_step,
+                     "peak_source": peak_src,
+                     "note": "per launch of rabit_gemv_mma_kernel, averaged over the launches of a step: algorithmic bytes of the "
+                             "step / device time of the step (launch gaps included); traffic = ncu dram bytes of the same launches"},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(sample_projections=n_proj)

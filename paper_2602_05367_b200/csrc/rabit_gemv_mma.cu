@@ -128,8 +128,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
+    unsigned int ns = 32;
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return; }
+        __nanosleep(ns);                                   // a waiting warp must not eat the issue slots of the working ones
+        if (ns < 256) ns *= 2;
     }
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
