@@ -107,9 +107,9 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
             if (!rabit_gemv_mma_supports(*layer, batch))
                 return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: integer-MMA GEMV cannot run batch %d", batch);
             e = cudaSuccess;
-            for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += 2)      // two batch rows share one pass over the weights
+            for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += rabit_gemv_mma_max_rows())   // up to 4 batch rows share one pass over the weights
                 e = rabit_launch_gemv_mma(*layer, (const char*)x + (size_t)b0 * G.N * 2, (char*)y + (size_t)b0 * G.M * 2,
-                                          batch - b0 >= 2 ? 2 : 1, st);
+                                          batch - b0 >= rabit_gemv_mma_max_rows() ? rabit_gemv_mma_max_rows() : batch - b0, st);
             break;
         case 3:
             if (!rabit_gemm_tc_supports(*layer, batch))
@@ -159,12 +159,13 @@ extern "C" int rabit_linear_group(const rabit_layer* const* layers, const void* 
     const void* xb[8];
     void* yb[8];
     cudaError_t e = cudaSuccess;
-    for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += 2) {            // two batch rows share one pass over the weights
+    const int rows = rabit_gemv_mma_max_rows();
+    for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += rows) {         // up to 4 batch rows share one pass over the weights
         for (int l = 0; l < n_layers; ++l) {
             xb[l] = (const char*)xs[l] + (size_t)b0 * layers[l]->geom.N * 2;
             yb[l] = (char*)ys[l] + (size_t)b0 * layers[l]->geom.M * 2;
         }
-        e = rabit_launch_gemv_mma_group(layers, n_layers, xb, yb, batch - b0 >= 2 ? 2 : 1, st);
+        e = rabit_launch_gemv_mma_group(layers, n_layers, xb, yb, batch - b0 >= rows ? rows : batch - b0, st);
     }
     if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear_group: launch failed: %s", cudaGetErrorString(e));
     return RABIT_OK;

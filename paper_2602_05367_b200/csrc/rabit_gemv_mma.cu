@@ -43,12 +43,23 @@
 namespace {
 
 constexpr int kMmaWarps = 8;
-constexpr int kBuildWarps = 2;
 constexpr int kMmaThreads = kMmaWarps * 32;
-constexpr int kThreads = (kMmaWarps + kBuildWarps) * 32;
 constexpr int kStageTiles = 16;
-constexpr int kRing = 8;
-constexpr int kHeadStages = kMmaWarps / kBuildWarps;    // first stages, built by the (still idle) MMA warps, one warp pair each
+constexpr int kHeadStages = kMmaWarps / 2;              // first stages, built by the (still idle) MMA warps, one warp pair each
+
+// Per batch width NB (rows of x handled in one pass over the weights): every A fragment feeds (NB+1)/2
+// MMAs (two batch rows each).  NB <= 2 runs two CTAs per SM; NB = 4 needs more registers (one CTA per SM)
+// and twice the builder warps (each pair converts half of the batch rows).  (NB = 8 would need 128
+// accumulator registers per thread and spills at this thread count, so a launch takes at most 4 rows.)
+template <int NB>
+struct Cfg {
+    static constexpr int kPairs = (NB + 1) / 2;
+    static constexpr int kBuildWarps = NB <= 2 ? 2 : 4;
+    static constexpr int kBuildRows = NB <= 2 ? NB : NB / 2;        // batch rows one builder lane converts
+    static constexpr int kThreads = (kMmaWarps + kBuildWarps) * 32;
+    static constexpr int kRing = NB <= 4 ? 8 : 6;
+    static constexpr int kMinBlocks = NB <= 2 ? 2 : 1;
+};
 constexpr int kBuildAhead = 3;                          // stages of raw x / h a builder lane keeps in flight
 constexpr long long kWaitLimitCycles = 1LL << 31;       // about one second
 constexpr unsigned int kSentinel = 0xFFFFFFFFu;         // resting content of the partial buffer ("not written yet")
@@ -93,17 +104,18 @@ struct GroupParams {
     int q, r;                // total_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
     FastDiv div_q, div_q1;   // by q, q + 1
     unsigned int* status;
+    int nb;                  // batch rows actually present (<= the kernel's NB); the others are neither read nor written
     GemvParams layer[kMaxGroup];
 };
 
 template <int NB>
 struct __align__(128) Smem {
-    uint4 bits[kRing][kStageTiles][32];
-    uint2 table[kRing][kStageTiles][NB * 16];           // word pair of lane l (n = l >> 2, tq = l & 3) at index l
-    int sum_t[kRing][kStageTiles][NB][4];               // sum of T over columns 8v .. 8v+7 of the tile, v = 0..3
+    uint4 bits[Cfg<NB>::kRing][kStageTiles][32];
+    uint2 table[Cfg<NB>::kRing][kStageTiles][NB * 16];  // batch row b, digit d, lane quad tq: pair index 16*b + 4*d + tq
+    int sum_t[Cfg<NB>::kRing][kStageTiles][NB][4];      // sum of T over columns 8v .. 8v+7 of the tile, v = 0..3
     float red[kMmaWarps][NB][RABIT_TILE_ROWS];
-    unsigned long long full[kRing];
-    unsigned long long empty[kRing];
+    unsigned long long full[Cfg<NB>::kRing];
+    unsigned long long empty[Cfg<NB>::kRing];
     unsigned int xmax_bits[NB];
     int abort_flag;
 };
@@ -117,6 +129,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -170,12 +185,60 @@ __device__ __forceinline__ void choose_scale(unsigned int xmax_bits, float hmax,
     inv = __int_as_float((127 - s) << 23);
 }
 
+
+// One lane's share of a stage: columns 8*bv .. +7 of tile j for ROWS batch rows starting at b0
+// -> digit words in fragment order + the sum of T over those columns.
+template <int NB, int ROWS>
+__device__ __forceinline__ void build_rows(Smem<NB>& S, int slot, int j, int bv, int kk, int b0, const uint4& hraw,
+                                           const uint4 (&xraw)[ROWS], const float (&sg_rows)[ROWS][RABIT_MAX_K]) {
+    const uint32_t hw[4] = {hraw.x, hraw.y, hraw.z, hraw.w};
+#pragma unroll
+    for (int rr = 0; rr < ROWS; ++rr) {
+        const float sg = kk == 0 ? sg_rows[rr][0] : (kk == 1 ? sg_rows[rr][1] : sg_rows[rr][2]);
+        const uint32_t xw[4] = {xraw[rr].x, xraw[rr].y, xraw[rr].z, xraw[rr].w};
+        int Tq[8];
+#pragma unroll
+        for (int c2 = 0; c2 < 4; ++c2) {
+            const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[c2]));
+            const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[c2]));
+            Tq[2 * c2] = __float2int_rn(hf.x * xf.x * sg);
+            Tq[2 * c2 + 1] = __float2int_rn(hf.y * xf.y * sg);
+        }
+        int tsum = 0;                        // |T| < 2^28, so eight of them fit
+#pragma unroll
+        for (int c = 0; c < 8; ++c) tsum += Tq[c];
+        uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][(b0 + rr) * 16]);
+#pragma unroll
+        for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
+            const int u = 2 * bv + hlf;
+            uint32_t X[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
+            const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
+            const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
+            uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
+            dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
+            dst[8] = __byte_perm(t0, t1, 0x7632);
+            dst[16] = __byte_perm(t2, t3, 0x5410);
+            dst[24] = __byte_perm(t2, t3, 0x7632);
+        }
+        S.sum_t[slot][j][b0 + rr][bv] = tsum;
+    }
+}
+
 template <int NB>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(Cfg<NB>::kThreads, Cfg<NB>::kMinBlocks)
 rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
+    constexpr int kRing = Cfg<NB>::kRing;
+    constexpr int kBuildWarps = Cfg<NB>::kBuildWarps;
+    constexpr int kBuildRows = Cfg<NB>::kBuildRows;
+    constexpr int kThreads = Cfg<NB>::kThreads;
+    constexpr int kPairs = Cfg<NB>::kPairs;
+    constexpr int kRed = (NB + 1) / 2;                   // (batch row, row) words one reducer thread owns: rows red_b0, red_b0 + 2, ...
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem<NB>& S = *reinterpret_cast<Smem<NB>*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nb = GP.nb;
     const int glo = range_lo(blockIdx.x, GP.q, GP.r);                      // this CTA's range in the launch's numbering
     const int ghi = range_lo(blockIdx.x + 1, GP.q, GP.r);
     volatile int* abort_flag = &S.abort_flag;
@@ -224,12 +287,14 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
                      tiles * RABIT_TILE_BYTES, bar);
         }
     }
-    // Builder lanes: lane index bi = 0..63 of the two builder warps takes tile bi >> 2 of every stage
-    // and columns 8*(bi & 3) .. +7 of it.
-    // The first kHeadStages stages are built by the MMA warps (pair warp >> 1 takes stage warp >> 1),
-    // which have nothing else to do until a table exists; the builder warps start behind them.
+    // Conversion lanes: lane index bi = 0..63 of a warp pair takes tile bi >> 2 of a stage and columns
+    // 8*(bi & 3) .. +7 of it.  The first kHeadStages stages are converted by the MMA warps (pair warp >> 1
+    // takes stage warp >> 1, all batch rows), which have nothing else to do until a table exists; the
+    // builder warps start behind them (with four builder warps each pair takes half of the batch rows).
     const int bi = ((warp & 1) << 5) | lane;
     const int bj = bi >> 2, bv = bi & 3;
+    const int bw = warp - kMmaWarps;
+    const int brow0 = (warp >= kMmaWarps && kBuildWarps == 4) ? (bw >> 1) * kBuildRows : 0;   // first batch row of a builder lane
     int pf_ct = 0, pf_k = 0;                          // (column tile, path) of the next prefetch / of the head stage
     int pf_stage = warp >= kMmaWarps ? kHeadStages : (warp >> 1);
     uint4 hq[kBuildAhead];
@@ -249,11 +314,11 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     int seg_end = min(n_tiles, (strip + 1) * C - lo);                       // relative to lo
     int rt = fdiv(strip, P.div_k);
     int k = strip - rt * G.K;
-    const int red_b = (tid >> 7) & 1, red_r = tid & 127;                   // (batch row, row) this thread reduces
-    const bool reducer = warp < kMmaWarps && red_b < NB;
+    const int red_b0 = (tid >> 7) & 1, red_r = tid & 127;                  // this thread reduces batch rows red_b0, red_b0 + 2, ... of row red_r
+    const bool reducer = warp < kMmaWarps && red_b0 < nb;
     float gval = 0.f;
     prefetch_h(0);                                   // builder: its first stage; MMA warp: its head stage
-    if (reducer && n_tiles > 0) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
+    if (reducer) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 
     if (first_pass) asm volatile("griddepcontrol.wait;" ::: "memory");
     first_pass = false;
@@ -265,7 +330,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     if (head_live) {
 #pragma unroll
         for (int b = 0; b < NB; ++b)
-            head_x[b] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
+            if (b < nb) head_x[b] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
     }
 
     // ---- largest |x| per batch row (fp16 bit patterns order like unsigned integers once the sign is cleared)
@@ -273,6 +338,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
         const int vec_per_row = G.N / 8;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
+            if (b >= nb) break;
             unsigned int m = 0;
             const uint4* xr = reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N);
             for (int i = tid; i < vec_per_row; i += kThreads) {
@@ -288,63 +354,29 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     }
     __syncthreads();
 
-    // One lane's share of a stage: columns 8*bv .. +7 of tile j, all batch rows -> digit words + sum of T.
-    auto build_part = [&](int slot, int j, int kk, const uint4& hraw, const uint4 (&xraw)[NB], const float (&sg_b)[NB][RABIT_MAX_K]) {
-        const uint32_t hw[4] = {hraw.x, hraw.y, hraw.z, hraw.w};
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const float sg = kk == 0 ? sg_b[b][0] : (kk == 1 ? sg_b[b][1] : sg_b[b][2]);
-            const uint32_t xw[4] = {xraw[b].x, xraw[b].y, xraw[b].z, xraw[b].w};
-            int Tq[8];
-#pragma unroll
-            for (int c2 = 0; c2 < 4; ++c2) {
-                const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[c2]));
-                const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[c2]));
-                Tq[2 * c2] = __float2int_rn(hf.x * xf.x * sg);
-                Tq[2 * c2 + 1] = __float2int_rn(hf.y * xf.y * sg);
-            }
-            int tsum = 0;                        // |T| < 2^28, so eight of them fit
-#pragma unroll
-            for (int c = 0; c < 8; ++c) tsum += Tq[c];
-            uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][b * 16]);
-#pragma unroll
-            for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
-                const int u = 2 * bv + hlf;
-                uint32_t X[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
-                const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
-                const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
-                uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
-                dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
-                dst[8] = __byte_perm(t0, t1, 0x7632);
-                dst[16] = __byte_perm(t2, t3, 0x5410);
-                dst[24] = __byte_perm(t2, t3, 0x7632);
-            }
-            S.sum_t[slot][j][b][bv] = tsum;
-        }
-    };
-    float sigma[NB][RABIT_MAX_K], sigma_inv[NB][RABIT_MAX_K];
-#pragma unroll
-    for (int b = 0; b < NB; ++b)
-#pragma unroll
-        for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-            choose_scale(S.xmax_bits[b], kk < G.K ? G.hmax[kk] : 0.f, sigma[b][kk], sigma_inv[b][kk]);
-
     if (warp >= kMmaWarps) {
-        // =========================== builder warps (and the copy issuers) ===========================
+        // =========================== builder warps (and the copy issuer) ===========================
         const int j = bj;
-        // a queue of kBuildAhead of this pair's stages of raw inputs hides the load latency
-        uint4 xq[kBuildAhead][NB];
+        float sg_rows[kBuildRows][RABIT_MAX_K];
+#pragma unroll
+        for (int rr = 0; rr < kBuildRows; ++rr)
+#pragma unroll
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
+                float inv;
+                choose_scale(S.xmax_bits[brow0 + rr], kk < G.K ? G.hmax[kk] : 0.f, sg_rows[rr][kk], inv);
+            }
+        // a queue of kBuildAhead stages of raw inputs hides the load latency
+        uint4 xq[kBuildAhead][kBuildRows];
         int kq[kBuildAhead];
         auto prefetch_x = [&](int d) {
             kq[d] = pf_k;
 #pragma unroll
-            for (int b = 0; b < NB; ++b) xq[d][b] = make_uint4(0u, 0u, 0u, 0u);
+            for (int rr = 0; rr < kBuildRows; ++rr) xq[d][rr] = make_uint4(0u, 0u, 0u, 0u);
             if (pf_stage < n_stages && pf_stage * kStageTiles + bj < n_tiles) {
 #pragma unroll
-                for (int b = 0; b < NB; ++b)
-                    xq[d][b] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)b * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
+                for (int rr = 0; rr < kBuildRows; ++rr)
+                    if (brow0 + rr < nb)
+                        xq[d][rr] = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)(brow0 + rr) * G.N + pf_ct * RABIT_TILE_COLS + 8 * bv));
             }
             pf_stage += 1;
             pf_ct += kStageTiles;
@@ -373,7 +405,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
                                  tiles * RABIT_TILE_BYTES, bar);
                     }
                 }
-                build_part(slot, j, kq[d], hq[d], xq[d], sigma);
+                build_rows<NB, kBuildRows>(S, slot, j, bv, kq[d], brow0, hq[d], xq[d], sg_rows);
                 prefetch_h(d);
                 prefetch_x(d);
                 __syncwarp();
@@ -384,22 +416,38 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     // ======================================= MMA warps =======================================
     const int gq = lane >> 2, tq = lane & 3;
     const int w = warp;
-    if (pf_stage < n_stages) {                // head stage of this warp pair (its slot's earlier use ended with the previous pass)
-        const int hslot = (it0 + pf_stage) % kRing;
-        if (head_live) build_part(hslot, bj, pf_k, hq[0], head_x, sigma);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.full[hslot]));
-    }
-    float sig_inv[RABIT_MAX_K];               // 1 / sigma of this thread's batch row at reduction time
+    float sig_inv[kRed][RABIT_MAX_K];         // 1 / sigma of the batch rows this thread reduces
+    {
+        float sg_all[NB][RABIT_MAX_K], inv_all[NB][RABIT_MAX_K];
 #pragma unroll
-    for (int kk = 0; kk < RABIT_MAX_K; ++kk) sig_inv[kk] = red_b < NB ? sigma_inv[red_b < NB ? red_b : 0][kk] : 1.f;
+        for (int b = 0; b < NB; ++b)
+#pragma unroll
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                choose_scale(S.xmax_bits[b], kk < G.K ? G.hmax[kk] : 0.f, sg_all[b][kk], inv_all[b][kk]);
+        if (pf_stage < n_stages) {            // head stage of this warp pair (its slot's earlier use ended with the previous pass)
+            const int hslot = (it0 + pf_stage) % kRing;
+            if (head_live) build_rows<NB, NB>(S, hslot, bj, bv, pf_k, 0, hq[0], head_x, sg_all);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_n(smem_u32(&S.full[hslot]), kBuildWarps / 2);
+        }
+#pragma unroll
+        for (int i = 0; i < kRed; ++i)
+#pragma unroll
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk) {
+                float v = inv_all[2 * i][kk];
+                if (2 * i + 1 < NB && red_b0) v = inv_all[2 * i + 1 < NB ? 2 * i + 1 : 0][kk];
+                sig_inv[i][kk] = v;
+            }
+    }
 
-    int acc[8][4];
+    int acc[kPairs][8][4];
     long long sum_t[NB];
 #pragma unroll
-    for (int p = 0; p < 8; ++p)
+    for (int jp = 0; jp < kPairs; ++jp)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[p][c] = 0;
+        for (int p = 0; p < 8; ++p)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[jp][p][c] = 0;
 #pragma unroll
     for (int b = 0; b < NB; ++b) sum_t[b] = 0;
     const int me = blockIdx.x;
@@ -420,30 +468,38 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
             st_f[b] = __ll2float_rn(t);
         }
 #pragma unroll
-        for (int p = 0; p < 8; ++p) {
+        for (int jp = 0; jp < kPairs; ++jp) {
+            const int b = 2 * jp + (tq >> 1);                                  // lanes tq = 0,1 hold batch row 2*jp, lanes 2,3 row 2*jp + 1
+            const float st = (2 * jp + 1 < NB && (tq >> 1)) ? st_f[2 * jp + 1 < NB ? 2 * jp + 1 : 0] : st_f[2 * jp];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const float lo2 = fmaf(256.f, (float)acc[p][2 * hf + 1], (float)acc[p][2 * hf]);
-                const float hi2 = __shfl_xor_sync(0xffffffffu, lo2, 1);        // digits 2,3 live in the odd lane
-                const int b = tq >> 1;
-                if ((tq & 1) == 0 && b < NB) {
-                    const float v = fmaf(65536.f, hi2, lo2);                    // 2^p * sum_j b T
-                    const float st = b == 0 ? st_f[0] : st_f[NB - 1];
-                    const float scale = __int_as_float((127 + 1 - p) << 23);    // 2^(1-p)
-                    S.red[w][b][16 * p + gq + 8 * hf] = fmaf(-scale, v, st);    // sum_j T - 2 sum_j b T
+            for (int p = 0; p < 8; ++p) {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const float lo2 = fmaf(256.f, (float)acc[jp][p][2 * hf + 1], (float)acc[jp][p][2 * hf]);
+                    const float hi2 = __shfl_xor_sync(0xffffffffu, lo2, 1);    // digits 2,3 live in the odd lane
+                    if ((tq & 1) == 0 && b < NB) {
+                        const float v = fmaf(65536.f, hi2, lo2);                // 2^p * sum_j b T
+                        const float scale = __int_as_float((127 + 1 - p) << 23);    // 2^(1-p)
+                        S.red[w][b][16 * p + gq + 8 * hf] = fmaf(-scale, v, st);    // sum_j T - 2 sum_j b T
+                    }
                 }
             }
         }
         bar_mma_warps();
         if (reducer) {
-            float sum = 0.f;
-#pragma unroll
-            for (int ww = 0; ww < kMmaWarps; ++ww) sum += S.red[ww][red_b][red_r];
-            const float inv = k == 0 ? sig_inv[0] : (k == 1 ? sig_inv[1] : sig_inv[2]);
-            unsigned int bits = __float_as_uint(gval * (sum * inv));
-            if (bits == kSentinel) bits = 0x7FFFFFFFu;                          // a NaN result must not look unwritten
             const size_t seg_id = (size_t)me + strip;
-            __stcg(reinterpret_cast<unsigned int*>(P.partial) + (seg_id * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r, bits);
+#pragma unroll
+            for (int i = 0; i < kRed; ++i) {
+                const int b = red_b0 + 2 * i;
+                if (b >= nb) break;
+                float sum = 0.f;
+#pragma unroll
+                for (int ww = 0; ww < kMmaWarps; ++ww) sum += S.red[ww][b][red_r];
+                const float inv = k == 0 ? sig_inv[i][0] : (k == 1 ? sig_inv[i][1] : sig_inv[i][2]);
+                unsigned int bits = __float_as_uint(gval * (sum * inv));
+                if (bits == kSentinel) bits = 0x7FFFFFFFu;                      // a NaN result must not look unwritten
+                __stcg(reinterpret_cast<unsigned int*>(P.partial) + (seg_id * RABIT_PARTIAL_BATCH + b) * RABIT_TILE_ROWS + red_r, bits);
+            }
         }
     };
 
@@ -455,34 +511,43 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
         gval = 0.f;
         if (reducer) gval = __half2float(P.g[(size_t)k * G.Mp + rt * RABIT_TILE_ROWS + red_r]);
 #pragma unroll
-        for (int p = 0; p < 8; ++p)
+        for (int jp = 0; jp < kPairs; ++jp)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc[p][c] = 0;
+            for (int p = 0; p < 8; ++p)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[jp][p][c] = 0;
 #pragma unroll
         for (int b = 0; b < NB; ++b) sum_t[b] = 0;
     };
 
-    // This warp's tiles are rel = w, w + 8, ...: the two of a stage are taken together when both lie in
-    // the current segment (the common case), which gives the scheduler two independent chains.
+    // One tile: 32 ANDs make the eight A fragments, each feeds kPairs MMAs (two batch rows each).
     auto one_tile = [&](int slot, int j) {
         const uint4 wv = S.bits[slot][j][lane];
-        uint2 bb = make_uint2(0u, 0u);
-        if (gq < 4 * NB) bb = S.table[slot][j][lane];
+        uint2 bb[kPairs];
+#pragma unroll
+        for (int jp = 0; jp < kPairs; ++jp) {
+            bb[jp] = make_uint2(0u, 0u);
+            if (2 * jp + (gq >> 2) < NB) bb[jp] = S.table[slot][j][jp * 32 + lane];
+        }
 #pragma unroll
         for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][j][b][lane & 3];   // this lane's quarter of the tile
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             const uint32_t mask = 0x01010101u << p;
-            mma_u8s8(acc[p], wv.x & mask, wv.y & mask, wv.z & mask, wv.w & mask, bb.x, bb.y);
+            const uint32_t a0 = wv.x & mask, a1 = wv.y & mask, a2 = wv.z & mask, a3 = wv.w & mask;
+#pragma unroll
+            for (int jp = 0; jp < kPairs; ++jp) mma_u8s8(acc[jp][p], a0, a1, a2, a3, bb[jp].x, bb[jp].y);
         }
     };
+    // This warp's tiles are rel = w, w + 8, ...: for NB <= 2 the two of a stage are taken together when both
+    // lie in the current segment (the common case), which gives the scheduler two independent chains.
 #pragma unroll 1
     for (int i = 0; i < n_stages; ++i) {
         const int slot = (it0 + i) % kRing;
         const int rel0 = i * kStageTiles + w, rel1 = rel0 + kMmaWarps;
         if (rel0 >= n_tiles) break;
         mbar_wait(smem_u32(&S.full[slot]), ((it0 + i) / kRing) & 1, abort_flag);
-        if (rel1 < seg_end) {
+        if (NB <= 2 && rel1 < seg_end) {
             const uint4 wa = S.bits[slot][w][lane];
             const uint4 wb = S.bits[slot][w + kMmaWarps][lane];
             uint2 ba = make_uint2(0u, 0u), bb = make_uint2(0u, 0u);
@@ -492,12 +557,12 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
 #pragma unroll
             for (int p = 0; p < 8; ++p) {
                 const uint32_t mask = 0x01010101u << p;
-                mma_u8s8(acc[p], wa.x & mask, wa.y & mask, wa.z & mask, wa.w & mask, ba.x, ba.y);
+                mma_u8s8(acc[0][p], wa.x & mask, wa.y & mask, wa.z & mask, wa.w & mask, ba.x, ba.y);
             }
 #pragma unroll
             for (int p = 0; p < 8; ++p) {
                 const uint32_t mask = 0x01010101u << p;
-                mma_u8s8(acc[p], wb.x & mask, wb.y & mask, wb.z & mask, wb.w & mask, bb.x, bb.y);
+                mma_u8s8(acc[0][p], wb.x & mask, wb.y & mask, wb.z & mask, wb.w & mask, bb.x, bb.y);
             }
         } else {
             while (rel0 >= seg_end) { segment_flush(); next_segment(); }
@@ -517,47 +582,50 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     }
 
     // ---- finish the row tiles whose last tile this CTA owns.  Every reducer thread works alone on its
-    //      (batch row, row): it reads that word of every contributor's partial, path by path and CTA by
-    //      CTA, waits (bounded) while a word still holds the sentinel, restores the sentinel for the next
-    //      call, adds in that fixed order and stores fp16.  No barrier and no fence is involved: a
-    //      partial word carries no other data with it.
+    //      (batch row, row) words: it reads that word of every contributor's partial, path by path and CTA
+    //      by CTA, waits (bounded) while a word still holds the sentinel, restores the sentinel for the next
+    //      call, adds in that fixed order and stores fp16.  No barrier and no fence is involved: a partial
+    //      word carries no other data with it.
     if (reducer) {
         constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
         for (int rt_f = fdiv(lo, P.div_kc); (rt_f + 1) * KC - 1 < lo + n_tiles; ++rt_f) {
-            float sum = 0.f;
 #pragma unroll 1
-            for (int kk = 0; kk < G.K; ++kk) {
-                const int s0 = (rt_f * G.K + kk) * C;
-                const int c0 = cta_of(P.base + s0, GP), c1 = cta_of(P.base + s0 + C - 1, GP);
-                unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
-                                    (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + red_b) * RABIT_TILE_ROWS + red_r;
+            for (int b = red_b0; b < nb; b += 2) {
+                float sum = 0.f;
 #pragma unroll 1
-                for (int c = c0; c <= c1; c += 8) {                            // eight loads in flight, consumed in order
-                    unsigned int v[8];
+                for (int kk = 0; kk < G.K; ++kk) {
+                    const int s0 = (rt_f * G.K + kk) * C;
+                    const int c0 = cta_of(P.base + s0, GP), c1 = cta_of(P.base + s0 + C - 1, GP);
+                    unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
+                                        (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + b) * RABIT_TILE_ROWS + red_r;
+#pragma unroll 1
+                    for (int c = c0; c <= c1; c += 8) {                        // eight loads in flight, consumed in order
+                        unsigned int v[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        v[u] = 0u;
-                        if (c + u <= c1) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (c + u > c1) break;
-                        if (v[u] == kSentinel) {
-                            const long long t0 = clock64();
-                            do {
-                                asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
-                                if (v[u] != kSentinel) break;
-                                if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
-                            } while (true);
+                        for (int u = 0; u < 8; ++u) {
+                            v[u] = 0u;
+                            if (c + u <= c1) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
                         }
-                        __stcg(src + u * kStride, kSentinel);
-                        sum += __uint_as_float(v[u]);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            if (c + u > c1) break;
+                            if (v[u] == kSentinel) {
+                                const long long t0 = clock64();
+                                do {
+                                    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
+                                    if (v[u] != kSentinel) break;
+                                    if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
+                                } while (true);
+                            }
+                            __stcg(src + u * kStride, kSentinel);
+                            sum += __uint_as_float(v[u]);
+                        }
+                        src += 8 * kStride;
                     }
-                    src += 8 * kStride;
                 }
+                const int row = rt_f * RABIT_TILE_ROWS + red_r;
+                if (row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(sum);
             }
-            const int row = rt_f * RABIT_TILE_ROWS + red_r;
-            if (row < G.M) P.y[(size_t)red_b * G.M + row] = __float2half_rn(sum);
         }
     }
     }                                                                          // MMA warps
@@ -594,7 +662,7 @@ static cudaError_t launch_nb(const GroupParams& GP, int grid, cudaStream_t strea
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(Cfg<NB>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -607,6 +675,9 @@ static cudaError_t launch_nb(const GroupParams& GP, int grid, cudaStream_t strea
 
 int rabit_gemv_mma_max_group() { return kMaxGroup; }
 
+// Largest number of batch rows one launch takes (the dispatcher walks the batch in such chunks).
+int rabit_gemv_mma_max_rows() { return 4; }
+
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch) {
     if (n_layers < 1 || n_layers > kMaxGroup || batch < 1 || batch > RABIT_MAX_GEMV_BATCH) return false;
     long long tiles = 0;
@@ -614,13 +685,15 @@ bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layer
     return tiles < (1LL << 31);
 }
 
-// One launch for n_layers independent layers, one or two batch rows (x_l: [batch][N_l], y_l: [batch][M_l]).
+// One launch for n_layers independent layers and 1..4 batch rows (x_l: [batch][N_l], y_l: [batch][M_l]).
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream) {
+    if (batch < 1 || batch > 4) return cudaErrorInvalidValue;
     GroupParams GP;
     GP.n_layers = n_layers;
     GP.total_tiles = 0;
     GP.status = layers[0]->d_status;
+    GP.nb = batch;
     for (int l = 0; l < n_layers; ++l) {
         const rabit_layer& L = *layers[l];
         GemvParams& P = GP.layer[l];
@@ -640,14 +713,16 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
     }
     for (int l = n_layers; l < kMaxGroup; ++l) GP.layer[l] = GP.layer[0];
     const int sms = layers[0]->sm_count > 0 ? layers[0]->sm_count : 148;
-    int grid = 2 * sms;                                      // two co-resident CTAs per SM
+    int grid = 2 * sms;                                      // NB <= 2: two co-resident CTAs per SM; NB > 2: two rounds of one
     if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
     if (grid > GP.total_tiles) grid = GP.total_tiles;
     GP.q = GP.total_tiles / grid;
     GP.r = GP.total_tiles % grid;
     GP.div_q = make_fastdiv((unsigned int)GP.q);
     GP.div_q1 = make_fastdiv((unsigned int)GP.q + 1u);
-    return batch == 1 ? launch_nb<1>(GP, grid, stream) : launch_nb<2>(GP, grid, stream);
+    if (batch == 1) return launch_nb<1>(GP, grid, stream);
+    if (batch == 2) return launch_nb<2>(GP, grid, stream);
+    return launch_nb<4>(GP, grid, stream);
 }
 
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {

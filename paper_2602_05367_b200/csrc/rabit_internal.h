@@ -44,6 +44,7 @@ cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
 bool rabit_gemv_mma_supports(const rabit_layer& L, int batch);
 int rabit_gemv_mma_max_group();
+int rabit_gemv_mma_max_rows();
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream);

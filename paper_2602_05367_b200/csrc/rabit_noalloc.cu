@@ -84,9 +84,10 @@ extern "C" int rabit_linear_static_scratch(const rabit_layer* layer, const void*
     view.d_flags = reinterpret_cast<unsigned int*>(base + plan.flags_off);
     view.d_status = reinterpret_cast<unsigned int*>(base + plan.status_off);
     cudaError_t e = cudaSuccess;
-    for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += 2)
+    const int rows = rabit_gemv_mma_max_rows();
+    for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += rows)
         e = rabit_launch_gemv_mma(view, (const char*)x + (size_t)b0 * G.N * 2, (char*)y + (size_t)b0 * G.M * 2,
-                                  batch - b0 >= 2 ? 2 : 1, st);
+                                  batch - b0 >= rows ? rows : batch - b0, st);
     if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear_static_scratch: launch failed: %s", cudaGetErrorString(e));
     return RABIT_OK;
 }
