@@ -713,7 +713,7 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
     }
     for (int l = n_layers; l < kMaxGroup; ++l) GP.layer[l] = GP.layer[0];
     const int sms = layers[0]->sm_count > 0 ? layers[0]->sm_count : 148;
-    int grid = 2 * sms;                                      // NB <= 2: two co-resident CTAs per SM; NB > 2: two rounds of one
+    int grid = (batch <= 2 ? 2 : 1) * sms;                   // as many CTAs as are resident at once (two per SM up to two batch rows)
     if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
     if (grid > GP.total_tiles) grid = GP.total_tiles;
     GP.q = GP.total_tiles / grid;
