@@ -91,6 +91,20 @@ RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16
                rabit_layer** out);
 
 /*
+ * Derive the sign planes from a full-precision weight on the device and pack them in one pass
+ * (Section 4.2, steps 1-3 / Algorithm 2: B_1 = sign(W), R_1 = W - g_1 (.) B_1 (.) h_1, B_2 = sign(R_1), ...;
+ * at the end of training these planes are frozen and W is discarded, end of Section 4.2):
+ *   W_dev   DEVICE fp32 [M][N] row-major, 16-byte aligned, not overlapping dev_buf
+ *   g, h    HOST fp16 bit patterns [K][M], [K][N] (the trained scales)
+ *   dev_buf, dev_bytes, stream, out   as rabit_pack
+ * The residual is kept in fp32; g*h is exact in fp32, so each update is one rounding; sign(0) = +1.
+ * The resulting layer is identical to rabit_pack of the planes that this recurrence yields.
+ * Streams W once (4 bytes per weight); returns after the work on `stream` has completed.
+ */
+RABIT_API int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uint16_t* h, int K, int M, int N,
+                      void* dev_buf, size_t dev_bytes, void* stream, rabit_layer** out);
+
+/*
  * Run the layer (Section 4.1 forward with the Eq. 2 weight):
  *   x  DEVICE fp16 [batch][N] row-major, 16-byte aligned
  *   y  DEVICE fp16 [batch][M] row-major, 16-byte aligned, must not overlap x

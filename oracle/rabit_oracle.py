@@ -102,24 +102,30 @@ def storage_bits_per_weight(K: int, M: int, N: int, scale_bits: int = 16) -> flo
     return (K * M * N + scale_bits * K * (M + N)) / float(M * N)
 
 
-def derive_planes(W: np.ndarray, g: np.ndarray, h: np.ndarray) -> np.ndarray:
+def derive_planes(W: np.ndarray, g: np.ndarray, h: np.ndarray, dtype=np.float64) -> np.ndarray:
     """Section 4.2 steps 1-3 / Algorithm 2: ``B_i = sign(R_{i-1})``, ``R_i = R_{i-1} - g_i*B_i*h_i``,
     ``R_0 = W``.  Returns canonical packed planes uint32 ``[K][M][N/32]``.
 
-    The paper does not define sign(0); the reading taken here is sign(0) = +1 (bit 0).
+    The paper does not define sign(0); the reading taken here is sign(0) = +1 (bit 0).  Nor does it
+    say in which precision the residual is kept.  A sign is an integer decided by floating point, so
+    a comparison with the CUDA path must decide it in the same precision: ``dtype=np.float32`` keeps
+    ``R`` in float32 and evaluates ``R - (g*B)*h`` with one rounding per update (``g*B`` and the
+    product of two float16 values are exact in float32), which is what the device kernel does.
+    The default float64 is the reference for everything else.
     """
-    W = np.asarray(W, dtype=np.float64)
-    g = np.asarray(g, dtype=np.float64)
-    h = np.asarray(h, dtype=np.float64)
+    W = np.asarray(W, dtype=dtype)
+    g = np.asarray(g, dtype=dtype)
+    h = np.asarray(h, dtype=dtype)
     K, M = g.shape
     N = h.shape[1]
     R = W.copy()
     planes = np.zeros((K, M, N // 32), dtype=np.uint32)
     weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    one = dtype(1.0)
     for k in range(K):
-        neg = R < 0.0                                          # bit 1 <=> sign -1
-        B = np.where(neg, -1.0, 1.0)
+        neg = R < 0                                            # bit 1 <=> sign -1
+        B = np.where(neg, -one, one).astype(dtype)
         words = (neg.reshape(M, N // 32, 32).astype(np.uint64) * weights).sum(axis=2)
         planes[k] = words.astype(np.uint32)
-        R = R - g[k][:, None] * B * h[k][None, :]
+        R = (R - (g[k][:, None] * B) * h[k][None, :]).astype(dtype)
     return planes

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     pack_host,
     unpack_host,
     rabit_pack,
+    rabit_derive_pack,
     rabit_linear,
     rabit_linear_group,
     rabit_linear_host,

@@ -38,6 +38,9 @@ def _load() -> ctypes.CDLL:
     lib.rabit_pack.restype = _c_int
     lib.rabit_pack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_size_t,
                                _c_void_p, ctypes.POINTER(_c_void_p)]
+    lib.rabit_derive_pack.restype = _c_int
+    lib.rabit_derive_pack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_size_t,
+                                      _c_void_p, ctypes.POINTER(_c_void_p)]
     lib.rabit_linear.restype = _c_int
     lib.rabit_linear.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
     lib.rabit_stage_bytes.restype = _c_size_t
@@ -178,6 +181,31 @@ def rabit_pack(planes, g, h, device="cuda:0", stream: Optional[int] = None) -> R
     with torch.cuda.device(dev):
         _check(_lib.rabit_pack(planes.ctypes.data, g16.ctypes.data, h16.ctypes.data, K, M, N,
                                _c_void_p(buf.data_ptr()), nbytes, _c_void_p(st), ctypes.byref(out)))
+    return RabitLayer(out.value, buf, K, M, N)
+
+
+def rabit_derive_pack(W, g, h, stream: Optional[int] = None) -> RabitLayer:
+    """Derive the sign planes of every path from the CUDA float32 weight W [M][N] and the fp16 scales
+    g [K][M], h [K][N] (host arrays) on the device, packed in place; returns the layer."""
+    import torch
+
+    if W.dtype != torch.float32 or not W.is_cuda or not W.is_contiguous() or W.dim() != 2:
+        raise ValueError("W must be a contiguous CUDA float32 matrix")
+    g16 = np.ascontiguousarray(g, dtype=np.float16).view(np.uint16)
+    h16 = np.ascontiguousarray(h, dtype=np.float16).view(np.uint16)
+    K, M = g16.shape
+    N = h16.shape[1]
+    if tuple(W.shape) != (M, N) or h16.shape[0] != K:
+        raise ValueError("inconsistent shapes between W, g and h")
+    nbytes = packed_bytes(K, M, N)
+    if nbytes == 0:
+        raise RabitError(-2, f"unsupported shape K={K} M={M} N={N}")
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    st = torch.cuda.current_stream(W.device).cuda_stream if stream is None else stream
+    out = _c_void_p()
+    with torch.cuda.device(W.device):
+        _check(_lib.rabit_derive_pack(_c_void_p(W.data_ptr()), g16.ctypes.data, h16.ctypes.data, K, M, N,
+                                      _c_void_p(buf.data_ptr()), nbytes, _c_void_p(st), ctypes.byref(out)))
     return RabitLayer(out.value, buf, K, M, N)
 
 

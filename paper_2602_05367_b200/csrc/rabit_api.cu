@@ -77,6 +77,64 @@ extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint1
     return RABIT_OK;
 }
 
+static bool ranges_overlap(const void* a, size_t an, const void* b, size_t bn);
+
+static void bind_layer(rabit_layer* L, const RabitGeom& G, const RabitHeader& hdr, void* dev_buf, int device) {
+    L->geom = G;
+    L->device = device;
+    L->variant = 0;
+    L->sm_count = 0;
+    cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, device);
+    L->dev_base = (char*)dev_buf;
+    L->dev_bytes = hdr.total_bytes;
+    L->d_bits = (const uint4*)(L->dev_base + hdr.off_bits);
+    L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
+    L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
+    L->d_partial = (float*)(L->dev_base + hdr.off_partial);
+    L->d_flags = (unsigned int*)(L->dev_base + hdr.off_flags);
+    L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
+}
+
+extern "C" int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uint16_t* h, int K, int M, int N,
+                                 void* dev_buf, size_t dev_bytes, void* stream, rabit_layer** out) {
+    rabit_clear_error();
+    if (!out) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: out is NULL");
+    *out = nullptr;
+    if (!W_dev || !g || !h || !dev_buf) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: null pointer");
+    if (((uintptr_t)dev_buf & 255u) != 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: dev_buf must be 256-byte aligned");
+    if (((uintptr_t)W_dev & 15u) != 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: W must be 16-byte aligned");
+    RabitGeom G;
+    RabitHeader hdr;
+    std::vector<uint8_t> tail;
+    try {
+        if (!rabit_build_meta(g, h, K, M, N, &G, &hdr, &tail))
+            return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_derive_pack: unsupported shape K=%d M=%d N=%d (need 1<=K<=3, M>=1, N%%32==0)", K, M, N);
+    } catch (const std::bad_alloc&) {
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: out of host memory");
+    }
+    if (dev_bytes < hdr.total_bytes)
+        return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_derive_pack: dev_buf holds %zu bytes, layer needs %zu", dev_bytes, (size_t)hdr.total_bytes);
+    cudaPointerAttributes attr;
+    RABIT_CUDA_TRY(cudaPointerGetAttributes(&attr, dev_buf));
+    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: dev_buf is not device memory");
+    if (ranges_overlap(W_dev, (size_t)M * N * 4, dev_buf, hdr.total_bytes))
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: W overlaps dev_buf");
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)dev_buf;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(base, &hdr, sizeof(hdr), cudaMemcpyHostToDevice, st));
+    RABIT_CUDA_TRY(cudaMemcpyAsync(base + hdr.off_g, tail.data(), tail.size(), cudaMemcpyHostToDevice, st));
+    cudaError_t e = rabit_launch_derive(G, W_dev, (const uint16_t*)(base + hdr.off_g), (const uint16_t*)(base + hdr.off_h),
+                                        (uint4*)(base + hdr.off_bits), st);
+    if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_derive_pack: launch failed: %s", cudaGetErrorString(e));
+    RABIT_CUDA_TRY(cudaStreamSynchronize(st));                       // the host staging buffers go out of scope
+    rabit_layer* L = new (std::nothrow) rabit_layer;
+    if (!L) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: out of host memory");
+    bind_layer(L, G, hdr, dev_buf, attr.device);
+    *out = L;
+    return RABIT_OK;
+}
+
 static bool ranges_overlap(const void* a, size_t an, const void* b, size_t bn) {
     uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
     return a0 < b0 + bn && b0 < a0 + an;

@@ -39,6 +39,15 @@ bool rabit_make_geom(int K, int M, int N, RabitGeom* out);          // hmax left
 void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr);
 bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out); // validates magic, version and shape
 
+// header + everything behind the sign tiles, for images whose tiles are written on the device (rabit_pack.cu)
+#ifdef __cplusplus
+#include <vector>
+bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* geom, RabitHeader* hdr,
+                      std::vector<uint8_t>* tail);
+#endif
+cudaError_t rabit_launch_derive(const RabitGeom& G, const float* W, const uint16_t* d_g, const uint16_t* d_h, uint4* d_tiles,
+                                cudaStream_t stream);
+
 // kernel launchers; each enqueues on `stream` and returns a cudaError_t from the launch
 cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);

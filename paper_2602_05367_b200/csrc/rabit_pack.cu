@@ -104,6 +104,34 @@ static void pack_tile(const RabitGeom& G, const uint32_t* plane /*[M][N/32]*/, i
     }
 }
 
+// Header and the sections behind the sign tiles (scales, resting partial buffer, reserved words, status)
+// for a layer whose tiles are produced elsewhere.  `tail` receives total_bytes - off_g bytes.
+bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* geom, RabitHeader* hdr,
+                      std::vector<uint8_t>* tail) {
+    RabitGeom G;
+    if (!rabit_make_geom(K, M, N, &G)) return false;
+    for (int k = 0; k < K; ++k) {
+        float m = 0.f;
+        for (int j = 0; j < N; ++j) {
+            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
+            if (m == m && (v > m || v != v)) m = v;
+        }
+        G.hmax[k] = m;
+    }
+    rabit_fill_header(G, hdr);
+    tail->assign((size_t)(hdr->total_bytes - hdr->off_g), 0);
+    uint8_t* base = tail->data() - hdr->off_g;                    // so that image offsets can be used
+    std::memset(base + hdr->off_partial, 0xFF, hdr->off_flags - hdr->off_partial);
+    uint16_t* gp = (uint16_t*)(base + hdr->off_g);
+    uint16_t* hp = (uint16_t*)(base + hdr->off_h);
+    for (int k = 0; k < K; ++k) {
+        std::memcpy(gp + (size_t)k * G.Mp, g + (size_t)k * M, (size_t)M * 2);
+        std::memcpy(hp + (size_t)k * N, h + (size_t)k * N, (size_t)N * 2);
+    }
+    *geom = G;
+    return true;
+}
+
 extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
                                int K, int M, int N, void* out, size_t out_bytes) {
     rabit_clear_error();

@@ -239,6 +239,37 @@ def test_derive_planes_brute_force():
     assert _sign(planes, 0, 2, 5) == 1.0
 
 
+def test_derive_planes_float32_mode_brute_force():
+    """The float32 mode (the device kernel's precision) against a scalar loop that rounds to float32 after
+    every update; inputs are fp16-valued scales and a float32 weight built so that the two precisions
+    disagree somewhere (residuals within float32 rounding of zero)."""
+    rng = np.random.default_rng(7)
+    K, M, N = 3, 6, 64
+    g = (np.abs(rng.standard_normal((K, M))) * np.array([1.0, 0.4, 0.15])[:, None]).astype(np.float16)
+    h = rng.uniform(0.5, 1.5, (K, N)).astype(np.float16)
+    W = rng.standard_normal((M, N)).astype(np.float32)
+    # a row whose first residual is an exact or near tie: W = g_0 * h_0 (+ one float32 ulp on odd columns)
+    tie = (g[0, 1].astype(np.float32) * h[0].astype(np.float32)).astype(np.float32)
+    W[1] = tie
+    W[1, 1::2] = np.nextafter(tie[1::2], np.float32(np.inf))
+    planes = orc.derive_planes(W, g, h, dtype=np.float32)
+    f32 = np.float32
+    for i in range(M):
+        for j in range(N):
+            r = f32(W[i, j])
+            for k in range(K):
+                neg = r < 0
+                assert _sign(planes, k, i, j) == (-1.0 if neg else 1.0)
+                gb = f32(-g[k, i]) if neg else f32(g[k, i])
+                r = f32(r - f32(gb * f32(h[k, j])))
+    # exact ties give residual +0 -> sign +1 in the next plane
+    assert all(_sign(planes, 1, 1, j) == 1.0 for j in range(0, N, 2))
+    # and float64 agrees wherever no residual comes within rounding of zero (all rows but the tie row)
+    p64 = orc.derive_planes(W.astype(np.float64), g, h)
+    keep = [i for i in range(M) if i != 1]
+    assert np.array_equal(planes[:, keep], p64[:, keep])
+
+
 def test_derived_paths_shrink_the_residual():
     """With the mean-magnitude scale each added path lowers ||W - W_hat||_F (error compensation)."""
     rng = np.random.default_rng(6)
