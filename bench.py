@@ -432,6 +432,62 @@ def bench_cases(args) -> dict:
             "gpu_launches": sum(c["copies"] for c in cases)}
 
 
+def bench_derive(args) -> dict:
+    """Extra workload: on-device derivation of the sign planes fused with packing (rabit_derive_pack) on the
+    7B-shaped weights; streams W (fp32) once, so the bound is HBM: 4 bytes in + K/8 bytes out per weight."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from synth import llama2_7b_layer_shapes
+
+    torch.cuda.set_device(0)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    cases = []
+    for sh in [s for i, s in enumerate(llama2_7b_layer_shapes()) if i in (0, 4, 6)]:
+        gen = torch.Generator(device="cuda"); gen.manual_seed(sh.M * 31 + sh.N)
+        Ws = [torch.randn((sh.M, sh.N), generator=gen, device="cuda", dtype=torch.float32) * 0.02 for _ in range(3)]   # 3 copies > L2
+        rng = np.random.default_rng(sh.M + sh.N)
+        h = rng.uniform(0.5, 1.5, (K_PATHS, sh.N)).astype(np.float16)
+        g = np.stack([rng.uniform(0.012, 0.02, sh.M), rng.uniform(0.005, 0.009, sh.M)]).astype(np.float16)
+        for W in Ws:
+            rabit.rabit_derive_pack(W, g, h).free()
+        reps = 4
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        # one call at a time, CUDA events around it (includes the upload of header and scales)
+        bufs = [torch.empty(rabit.packed_bytes(K_PATHS, sh.M, sh.N), dtype=torch.uint8, device="cuda") for _ in Ws]
+        from paper_2602_05367_b200 import binding
+        import ctypes
+        lib, vp = binding.raw_lib(), ctypes.c_void_p
+        g16, h16 = g.view(np.uint16), h.view(np.uint16)
+        st = torch.cuda.current_stream().cuda_stream
+        handles = []
+        ev0.record()
+        for r in range(reps):
+            for W, buf in zip(Ws, bufs):
+                out = vp()
+                rc = lib.rabit_derive_pack(vp(W.data_ptr()), g16.ctypes.data, h16.ctypes.data, K_PATHS, sh.M, sh.N,
+                                           vp(buf.data_ptr()), buf.numel(), vp(st), ctypes.byref(out))
+                assert rc == 0, rabit.last_error()
+                handles.append(out)
+        ev1.record(); torch.cuda.synchronize()
+        for hnd in handles:
+            lib.rabit_free(hnd)
+        us = ev0.elapsed_time(ev1) * 1e3 / (reps * len(Ws))
+        nbytes = 4 * sh.M * sh.N + K_PATHS * sh.M * sh.N // 8 + 2 * K_PATHS * (sh.M + sh.N)
+        cases.append({"M": sh.M, "N": sh.N, "us": us, "gbs": nbytes / us / 1e3,
+                      "roofline": {"bound": "hbm", "achieved": nbytes / us / 1e3, "peak": hbm_peak, "unit": "GB/s", "frac": nbytes / us / 1e3 / hbm_peak},
+                      "note": "back-to-back asynchronous calls through the C ABI, CUDA events around all of them: includes the "
+                              "upload of header and scales and two fills per call"})
+        del Ws
+        torch.cuda.empty_cache()
+    head = max(cases, key=lambda c: c["M"] * c["N"])
+    return {"metric": "sign-plane derivation + packing GB/s", "value": head["gbs"], "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": 3, "ms_per_step": head["us"] / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": {"workload": "derive7b", "K": K_PATHS}, "cases": cases,
+            "roofline": head["roofline"], "gpu_launches": len(cases) * 12}
+
+
 def bench_reference(args) -> dict:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -468,13 +524,15 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-group", action="store_true", help="one rabit_linear launch per projection (7 per step instead of 4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemv70b", "sweep8b"],
+    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemv70b", "sweep8b", "derive7b"],
                     help="decoder7b is the contract's line; the others are extra single-GPU measurements")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         res = bench_reference(args)
+    elif args.workload == "derive7b":
+        res = bench_derive(args)
     elif args.workload != "decoder7b":
         res = bench_cases(args)
     else:

@@ -99,7 +99,9 @@ RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16
  *   dev_buf, dev_bytes, stream, out   as rabit_pack
  * The residual is kept in fp32; g*h is exact in fp32, so each update is one rounding; sign(0) = +1.
  * The resulting layer is identical to rabit_pack of the planes that this recurrence yields.
- * Streams W once (4 bytes per weight); returns after the work on `stream` has completed.
+ * Streams W once (4 bytes per weight).  Asynchronous on `stream`: g and h are read before the call
+ * returns, W when the kernel runs; the layer may be used by later work on the same stream (or after a
+ * synchronisation on any stream).
  */
 RABIT_API int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uint16_t* h, int K, int M, int N,
                       void* dev_buf, size_t dev_bytes, void* stream, rabit_layer** out);

@@ -123,11 +123,15 @@ extern "C" int rabit_derive_pack(const float* W_dev, const uint16_t* g, const ui
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)dev_buf;
     RABIT_CUDA_TRY(cudaMemcpyAsync(base, &hdr, sizeof(hdr), cudaMemcpyHostToDevice, st));
+    // scales from the host (a few KB), the scratch sections by device-side fills
     RABIT_CUDA_TRY(cudaMemcpyAsync(base + hdr.off_g, tail.data(), tail.size(), cudaMemcpyHostToDevice, st));
+    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_partial, 0xFF, (size_t)(hdr.off_flags - hdr.off_partial), st));
+    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_flags, 0, (size_t)(hdr.total_bytes - hdr.off_flags), st));
     cudaError_t e = rabit_launch_derive(G, W_dev, (const uint16_t*)(base + hdr.off_g), (const uint16_t*)(base + hdr.off_h),
                                         (uint4*)(base + hdr.off_bits), st);
     if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_derive_pack: launch failed: %s", cudaGetErrorString(e));
-    RABIT_CUDA_TRY(cudaStreamSynchronize(st));                       // the host staging buffers go out of scope
+    // No synchronisation: copies from pageable host memory return once the source has been staged, so the
+    // local buffers may go out of scope; the layer is usable by later work on the same stream.
     rabit_layer* L = new (std::nothrow) rabit_layer;
     if (!L) return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: out of host memory");
     bind_layer(L, G, hdr, dev_buf, attr.device);

@@ -39,7 +39,7 @@ bool rabit_make_geom(int K, int M, int N, RabitGeom* out);          // hmax left
 void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr);
 bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out); // validates magic, version and shape
 
-// header + everything behind the sign tiles, for images whose tiles are written on the device (rabit_pack.cu)
+// header + scale sections, for images whose tiles are written on the device (rabit_pack.cu)
 #ifdef __cplusplus
 #include <vector>
 bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* geom, RabitHeader* hdr,

@@ -104,8 +104,8 @@ static void pack_tile(const RabitGeom& G, const uint32_t* plane /*[M][N/32]*/, i
     }
 }
 
-// Header and the sections behind the sign tiles (scales, resting partial buffer, reserved words, status)
-// for a layer whose tiles are produced elsewhere.  `tail` receives total_bytes - off_g bytes.
+// Header and the two scale sections for a layer whose tiles are produced elsewhere.
+// `tail` receives off_partial - off_g bytes (the image from off_g up to the scratch sections).
 bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* geom, RabitHeader* hdr,
                       std::vector<uint8_t>* tail) {
     RabitGeom G;
@@ -119,9 +119,8 @@ bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N,
         G.hmax[k] = m;
     }
     rabit_fill_header(G, hdr);
-    tail->assign((size_t)(hdr->total_bytes - hdr->off_g), 0);
+    tail->assign((size_t)(hdr->off_partial - hdr->off_g), 0);
     uint8_t* base = tail->data() - hdr->off_g;                    // so that image offsets can be used
-    std::memset(base + hdr->off_partial, 0xFF, hdr->off_flags - hdr->off_partial);
     uint16_t* gp = (uint16_t*)(base + hdr->off_g);
     uint16_t* hp = (uint16_t*)(base + hdr->off_h);
     for (int k = 0; k < K; ++k) {
