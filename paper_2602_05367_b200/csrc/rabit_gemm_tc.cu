@@ -25,23 +25,25 @@
 namespace {
 
 constexpr int kTileM = 128;                 // weight rows per output tile
-constexpr int kTileB = 256;                 // batch rows per output tile (MMA N)
+// batch rows per output tile (MMA N) and paths: TB = 256 with up to 2 paths or TB = 128 with 3 (template parameters):
+// paths x TB accumulator columns must fit the 512 columns of tensor memory
 constexpr int kStepCols = 64;               // input columns per pipeline step (128 bytes of fp16: one swizzle row)
 constexpr int kStages = 3;
-constexpr int kMaxPaths = 2;                // accumulators of 256 columns: 2 x 256 = the 512 columns of tensor memory
 constexpr int kExpandWarps = 8;
 constexpr int kThreads = (2 + kExpandWarps) * 32;
 constexpr long long kWaitLimitCycles = 1LL << 31;
 
+template <int TB, int KP>
 struct __align__(1024) Stage {
-    __half a[kMaxPaths][kTileM * kStepCols];          // 2 x 16 KB, +-h, swizzled
-    __half x[kTileB * kStepCols];                     // 32 KB, swizzled by TMA
-    uint4 bits[kMaxPaths][2][32];                     // packed sign tiles: 2 column tiles per step per path
-    __half h[kMaxPaths][kStepCols];
+    __half a[KP][kTileM * kStepCols];                 // 16 KB per path, +-h, swizzled
+    __half x[TB * kStepCols];                         // 32 or 16 KB, swizzled by TMA
+    uint4 bits[KP][2][32];                            // packed sign tiles: 2 column tiles per step per path
+    __half h[KP][kStepCols];
 };
 
+template <int TB, int KP>
 struct Smem {
-    Stage stage[kStages];
+    Stage<TB, KP> stage[kStages];
     unsigned long long full[kStages];                 // TMA bytes landed (x, bits, h)
     unsigned long long a_ready[kStages];              // expanders done
     unsigned long long empty[kStages];                // MMAs that read the stage retired
@@ -105,9 +107,9 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;                        // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: D fp32, A and B fp16, both K-major, N = 256, M = 128.
-__device__ __forceinline__ uint32_t umma_idesc() {
-    return (1u << 4) | ((uint32_t)(kTileB >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+// Instruction descriptor: D fp32, A and B fp16, both K-major, N = batch tile, M = 128.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
@@ -126,8 +128,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                  : "r"(taddr) : "memory");
 }
 
+template <int TB, int KP>
 __global__ void __launch_bounds__(kThreads, 1)
 rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_map) {
+    using Stage = Stage<TB, KP>;
+    using Smem = Smem<TB, KP>;
+    constexpr int kTileB = TB;
+    constexpr int kMaxPaths = KP;
     extern __shared__ unsigned char smem_raw[];
     // the swizzled operand tiles need 1024-byte alignment; the launch reserves the slack
     Smem& S = *reinterpret_cast<Smem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
@@ -183,7 +190,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     } else if (warp == 1) {
         // ===================================== MMA issuer =====================================
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc();
+            const uint32_t idesc = umma_idesc(kTileB);
             int it = 0, tile_i = 0;
             for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
                 if (tile_i > 0) mbar_wait(smem_u32(&S.acc_empty), (tile_i - 1) & 1, abort_flag);   // epilogue has drained the accumulators
@@ -212,7 +219,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int e = warp - 2;                               // 0..7
         const int et = e * 32 + lane;                         // 0..255
         const int quarter = warp & 3;                         // tensor-memory lanes this warp may read: 32*quarter .. +31
-        const int col_half = e >> 2;                          // which 128 of the 256 batch columns this warp drains
+        const int col_half = e >> 2;                          // which half of the tile's batch columns this warp drains
         int it = 0, tile_i = 0;
         for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
@@ -258,18 +265,24 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
 #pragma unroll
             for (int k = 0; k < kMaxPaths; ++k) gk[k] = (k < K && row < G.Mp) ? __half2float(P.g[(size_t)k * G.Mp + row]) : 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < 128; c0 += 32) {
-                const int col = col_half * 128 + c0;
-                uint32_t d0[32], d1[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, d0);
-                if (K > 1) tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(kTileB + col), d1);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            for (int c0 = 0; c0 < kTileB / 2; c0 += 32) {
+                const int col = col_half * (kTileB / 2) + c0;
+                float v[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] = 0.f;
+#pragma unroll
+                for (int k = 0; k < kMaxPaths; ++k) {
+                    if (k >= K) break;
+                    uint32_t d[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(k * kTileB + col), d);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) v[c] = fmaf(gk[k], __uint_as_float(d[c]), v[c]);
+                }
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    float v = gk[0] * __uint_as_float(d0[c]);
-                    if (K > 1) v = fmaf(gk[1], __uint_as_float(d1[c]), v);
                     const int b = bt * kTileB + col + c;
-                    if (b < P.batch && row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(v);
+                    if (b < P.batch && row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(v[c]);
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -308,16 +321,17 @@ EncodeTiledFn encode_tiled_fn() {
 }  // namespace
 
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch) {
-    return batch > RABIT_MAX_GEMV_BATCH && L.geom.K <= kMaxPaths && encode_tiled_fn() != nullptr;
+    return batch > RABIT_MAX_GEMV_BATCH && L.geom.K <= 3 && encode_tiled_fn() != nullptr;
 }
 
-cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
+template <int TB, int KP>
+static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)L.geom.N, (cuuint64_t)batch};
     const cuuint64_t strides[1] = {(cuuint64_t)L.geom.N * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kStepCols, (cuuint32_t)kTileB};
+    const cuuint32_t box[2] = {(cuuint32_t)kStepCols, (cuuint32_t)TB};
     const cuuint32_t estr[2] = {1, 1};
     if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -331,17 +345,22 @@ cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, i
     P.y = (__half*)y;
     P.status = L.d_status;
     P.batch = batch;
-    P.n_bt = (batch + kTileB - 1) / kTileB;
+    P.n_bt = (batch + TB - 1) / TB;
     P.n_tiles = L.geom.n_rt * P.n_bt;
     static bool attr_done = false;
-    const size_t smem = sizeof(Smem) + 1024;                       // slack for the 1024-byte alignment of the stages
+    const size_t smem = sizeof(Smem<TB, KP>) + 1024;               // slack for the 1024-byte alignment of the stages
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel<TB, KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     int grid = L.sm_count > 0 ? L.sm_count : 148;
     if (grid > P.n_tiles) grid = P.n_tiles;
-    rabit_gemm_tc_kernel<<<grid, kThreads, smem, stream>>>(P, map);
+    rabit_gemm_tc_kernel<TB, KP><<<grid, kThreads, smem, stream>>>(P, map);
     return cudaGetLastError();
+}
+
+cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
+    if (L.geom.K <= 2) return launch_gemm<256, 2>(L, x, y, batch, stream);
+    return launch_gemm<128, 3>(L, x, y, batch, stream);              // three accumulators of 128 columns
 }

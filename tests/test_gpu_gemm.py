@@ -18,6 +18,8 @@ GEMM = 3    # variant number of the tcgen05 GEMM
     (2, 1000, 1184, 300),    # several row tiles, two batch tiles with a ragged tail, N % 64 == 32
     (2, 384, 2048, 512),
     (2, 2500, 512, 257),
+    (3, 300, 352, 130),      # three paths: 128-wide batch tiles, two of them with a ragged tail
+    (3, 128, 64, 17),
 ])
 @pytest.mark.parametrize("variant", [0, GEMM])
 def test_gemm_shapes(K, M, N, batch, variant):
@@ -51,8 +53,9 @@ def test_gemm_structured_inputs():
     assert not y.any()
 
 
-def test_three_paths_large_batch_falls_back():
-    """K = 3 does not fit the tensor-memory accumulators; the dispatcher must still give the right answer."""
+def test_three_paths_large_batch():
+    """K = 3 runs with three 128-column accumulators; automatic dispatch and the explicit variant agree with the oracle."""
     L = make_layer(160, 256, 3, key=(63,))
     x = make_x(48, 256, key=(63,))
     check_against_oracle(L, x, run_layer(L, x, 0))
+    check_against_oracle(L, x, run_layer(L, x, GEMM))
