@@ -10,10 +10,10 @@
 //
 // One CTA per SM, persistent over output tiles of 128 weight rows x 256 batch rows:
 //   warp 0      producer: per 64-column step, one TMA tile of x (128B swizzle) plus bulk copies of
-//               the packed sign tiles and the h slices of that step, into a 3-stage ring
+//               the packed sign tiles and the h slices of that step, into a ring of up to 8 steps
 //   warp 1      allocates tensor memory, issues tcgen05.mma (M=128, N=256, K=16, kind::f16) for every
 //               path into that path's accumulator, commits stages back to the producer
-//   warps 2..9  expand packed signs to +-h fp16 in the canonical K-major 128B-swizzled layout, then
+//   warps 2..9  expand packed signs to +-h fp16 in the canonical K-major 128B-swizzled layout (two A stages), then
 //               (same warps) read the accumulators with tcgen05.ld for the epilogue
 // Every wait is bounded; on a time-out the CTA sets the status word, skips the remaining waits,
 // frees its tensor memory and returns.
@@ -28,25 +28,40 @@ constexpr int kTileM = 128;                 // weight rows per output tile
 // batch rows per output tile (MMA N) and paths: TB = 256 with up to 2 paths or TB = 128 with 3 (template parameters):
 // paths x TB accumulator columns must fit the 512 columns of tensor memory
 constexpr int kStepCols = 64;               // input columns per pipeline step (128 bytes of fp16: one swizzle row)
-constexpr int kStages = 3;
+constexpr int kAStages = 2;                 // expanded A tiles are double-buffered
 constexpr int kExpandWarps = 8;
 constexpr int kThreads = (2 + kExpandWarps) * 32;
 constexpr long long kWaitLimitCycles = 1LL << 31;
 
+// What the copy engine brings per 64-column step (deep ring: it hides the global-memory latency) ...
 template <int TB, int KP>
-struct __align__(1024) Stage {
-    __half a[KP][kTileM * kStepCols];                 // 16 KB per path, +-h, swizzled
-    __half x[TB * kStepCols];                         // 32 or 16 KB, swizzled by TMA
+struct __align__(1024) InStage {
+    __half x[TB * kStepCols];                         // 8..32 KB, swizzled by TMA
     uint4 bits[KP][2][32];                            // packed sign tiles: 2 column tiles per step per path
     __half h[KP][kStepCols];
+};
+// ... and what the expander warps make of it (two steps: one being multiplied, one being written).
+template <int KP>
+struct __align__(1024) AStage {
+    __half a[KP][kTileM * kStepCols];                 // 16 KB per path, +-h, swizzled
+};
+
+// Input-ring depth: as many steps as fit beside the A ring in 222 KB, at most 8.
+template <int TB, int KP>
+struct GemmCfg {
+    static constexpr int kInBytes = (int)sizeof(InStage<TB, KP>);
+    static constexpr int kFit = (222 * 1024 - kAStages * (int)sizeof(AStage<KP>)) / kInBytes;
+    static constexpr int kStages = kFit > 8 ? 8 : kFit;
 };
 
 template <int TB, int KP>
 struct Smem {
-    Stage<TB, KP> stage[kStages];
-    unsigned long long full[kStages];                 // TMA bytes landed (x, bits, h)
-    unsigned long long a_ready[kStages];              // expanders done
-    unsigned long long empty[kStages];                // MMAs that read the stage retired
+    AStage<KP> astage[kAStages];
+    InStage<TB, KP> stage[GemmCfg<TB, KP>::kStages];
+    unsigned long long full[8];                       // TMA bytes landed (x, bits, h)
+    unsigned long long empty[8];                      // MMAs that read the input stage retired
+    unsigned long long a_ready[kAStages];             // expanders done
+    unsigned long long a_empty[kAStages];             // MMAs that read the A stage retired
     unsigned long long acc_ready;                     // all MMAs of the tile retired
     unsigned long long acc_empty;                     // epilogue has read the accumulators
     uint32_t tmem_base;
@@ -131,8 +146,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 template <int TB, int KP>
 __global__ void __launch_bounds__(kThreads, 1)
 rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_map) {
-    using Stage = Stage<TB, KP>;
+    using Stage = InStage<TB, KP>;
     using Smem = Smem<TB, KP>;
+    constexpr int kStages = GemmCfg<TB, KP>::kStages;
     constexpr int kTileB = TB;
     constexpr int kMaxPaths = KP;
     extern __shared__ unsigned char smem_raw[];
@@ -147,8 +163,11 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&S.full[s]), 1);
-            mbar_init(smem_u32(&S.a_ready[s]), kExpandWarps);
             mbar_init(smem_u32(&S.empty[s]), 1);
+        }
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(smem_u32(&S.a_ready[s]), kExpandWarps);
+            mbar_init(smem_u32(&S.a_empty[s]), 1);
         }
         mbar_init(smem_u32(&S.acc_ready), 1);
         mbar_init(smem_u32(&S.acc_empty), kExpandWarps);
@@ -196,20 +215,21 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                 if (tile_i > 0) mbar_wait(smem_u32(&S.acc_empty), (tile_i - 1) & 1, abort_flag);   // epilogue has drained the accumulators
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int s = 0; s < n_steps; ++s, ++it) {
-                    const int slot = it % kStages;
+                    const int slot = it % kStages, aslot = it % kAStages;
                     mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
-                    mbar_wait(smem_u32(&S.a_ready[slot]), (it / kStages) & 1, abort_flag);
+                    mbar_wait(smem_u32(&S.a_ready[aslot]), (it / kAStages) & 1, abort_flag);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     Stage& st = S.stage[slot];
                     const int ksub = min(2, G.n_ct - 2 * s) * 2;                                   // MMAs of K = 16 in this step (2 per column tile)
                     const uint64_t bdesc = umma_desc(smem_u32(st.x));
                     for (int k = 0; k < K; ++k) {
-                        const uint64_t adesc = umma_desc(smem_u32(st.a[k]));
+                        const uint64_t adesc = umma_desc(smem_u32(S.astage[aslot].a[k]));
                         for (int kk = 0; kk < ksub; ++kk)
                             umma_f16(tmem_base + (uint32_t)k * kTileB, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc,
                                      (s > 0 || kk > 0) ? 1u : 0u);
                     }
-                    umma_commit(smem_u32(&S.empty[slot]));                                         // frees the stage when these MMAs retire
+                    umma_commit(smem_u32(&S.empty[slot]));                                         // frees both stages when these MMAs retire
+                    umma_commit(smem_u32(&S.a_empty[aslot]));
                 }
                 umma_commit(smem_u32(&S.acc_ready));
             }
@@ -220,42 +240,46 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int et = e * 32 + lane;                         // 0..255
         const int quarter = warp & 3;                         // tensor-memory lanes this warp may read: 32*quarter .. +31
         const int col_half = e >> 2;                          // which half of the tile's batch columns this warp drains
+        // expander role of this thread, the same in every step: one packed word position per path
+        const int x_ct2 = et >> 7, x_l = (et >> 2) & 31, x_a = et & 3;
+        const int x_gq = x_l >> 2, x_tq = x_l & 3;
+        const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
+        const uint32_t x_aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
         int it = 0, tile_i = 0;
         for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
             for (int s = 0; s < n_steps; ++s, ++it) {
-                const int slot = it % kStages;
+                const int slot = it % kStages, aslot = it % kAStages;
                 mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
+                if (it >= kAStages) mbar_wait(smem_u32(&S.a_empty[aslot]), ((it / kAStages) - 1) & 1, abort_flag);
                 Stage& st = S.stage[slot];
+                AStage<KP>& ast = S.astage[aslot];
                 const int cts = min(2, G.n_ct - 2 * s);
-                // packed words of the step: [path][column tile][lane][word a]; 256 threads take them round-robin
-                for (int wi = et; wi < K * 2 * 128; wi += kExpandWarps * 32) {
-                    const int k = wi >> 8, ct2 = (wi >> 7) & 1, l = (wi >> 2) & 31, a = wi & 3;
-                    const int gq = l >> 2, tq = l & 3;
+                // This thread's packed word (column tile ct2, lane l, word a) of every path: rows 16*p + gq + 8*(a&1),
+                // columns 32*ct2 + 16*(a>>1) + 4*tq + c (c = 0..3) = bytes 0..7 of 16-byte chunk 4*ct2 + 2*(a>>1) + (tq>>1)
+                // of the row (second half if tq is odd); the chunk is XOR-swizzled with the row.
+#pragma unroll
+                for (int k = 0; k < kMaxPaths; ++k) {
+                    if (k >= K) break;
                     uint32_t w = 0;
                     uint2 hv = make_uint2(0u, 0u);
-                    if (ct2 < cts) {
-                        w = reinterpret_cast<const uint32_t*>(&st.bits[k][ct2][l])[a];
-                        hv = *reinterpret_cast<const uint2*>(&st.h[k][32 * ct2 + 16 * (a >> 1) + 4 * tq]);
+                    if (x_ct2 < cts) {
+                        w = reinterpret_cast<const uint32_t*>(&st.bits[k][x_ct2][x_l])[x_a];
+                        hv = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff]);
                     }
-                    // columns 32*ct2 + 16*(a>>1) + 4*tq + c (c = 0..3) = bytes 0..7 of 16-byte chunk number
-                    // 4*ct2 + 2*(a>>1) + (tq>>1) in the row, second half if tq is odd; rows 16*p + gq + 8*(a&1)
-                    const int chunk = 4 * ct2 + 2 * (a >> 1) + (tq >> 1);
-                    unsigned char* base = reinterpret_cast<unsigned char*>(st.a[k]) + (gq + 8 * (a & 1)) * 128 + ((chunk ^ gq) << 4) + 8 * (tq & 1);
+                    const uint32_t u01 = __byte_perm(w, 0u, 0x1404);                       // bytes [0, c0, 0, c1]: bit p of a column -> bit 8+p / 24+p
+                    const uint32_t u23 = __byte_perm(w, 0u, 0x3424);                       // bytes [0, c2, 0, c3]
+                    const uint32_t dst = smem_u32(ast.a[k]) + x_aoff;
 #pragma unroll
                     for (int p = 0; p < 8; ++p) {
-                        const uint32_t sh = w << (7 - p);                                  // bit p of every byte -> bit 7
-                        const uint32_t s01 = __byte_perm(sh, 0u, 0x1404);                  // bytes [0, c0, 0, c1]
-                        const uint32_t s23 = __byte_perm(sh, 0u, 0x3424);                  // bytes [0, c2, 0, c3]
-                        uint2 o;
-                        o.x = hv.x ^ (s01 & 0x80008000u);                                  // flip the fp16 sign where the weight is -1
-                        o.y = hv.y ^ (s23 & 0x80008000u);
-                        *reinterpret_cast<uint2*>(base + p * 16 * 128) = o;
+                        const uint32_t ox = hv.x ^ ((u01 << (7 - p)) & 0x80008000u);       // flip the fp16 sign where the weight is -1
+                        const uint32_t oy = hv.y ^ ((u23 << (7 - p)) & 0x80008000u);
+                        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(ox), "r"(oy) : "memory");
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");              // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&S.a_ready[slot]));
+                if (lane == 0) mbar_arrive(smem_u32(&S.a_ready[aslot]));
             }
             // ---- epilogue of this tile
             mbar_wait(smem_u32(&S.acc_ready), tile_i & 1, abort_flag);
@@ -361,6 +385,8 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
 }
 
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
-    if (L.geom.K <= 2) return launch_gemm<256, 2>(L, x, y, batch, stream);
-    return launch_gemm<128, 3>(L, x, y, batch, stream);              // three accumulators of 128 columns
+    if (L.geom.K > 2) return launch_gemm<128, 3>(L, x, y, batch, stream);          // three accumulators of 128 columns
+    // Always the widest batch tile: a tcgen05.mma of M = 128 takes about 128 clocks whatever its N (measured),
+    // so narrower tiles would not shorten a step, they would only expand the signs more often.
+    return launch_gemm<256, 2>(L, x, y, batch, stream);
 }
