@@ -173,6 +173,22 @@ RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, vo
  */
 RABIT_API int rabit_linear_static_scratch(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
+/*
+ * Health of a layer's kernels.  Every wait inside the kernels is bounded (about one second); a wait that
+ * runs out makes the kernel set the layer's status word, skip its remaining waits and return, so the
+ * context stays usable but the outputs of that call are invalid.  This call synchronises `stream`, reads
+ * the word and returns RABIT_OK or RABIT_DEVICE_FAULT (the word is cleared when `clear` is non-zero).
+ */
+RABIT_API int rabit_layer_status(const rabit_layer* layer, int clear, void* stream);
+
+/*
+ * Self-test of the bounded-wait mechanism: launches one tiny kernel that waits on a barrier nobody will
+ * ever signal, with a limit of `limit_us` microseconds (1..100000), and reports whether the kernel gave
+ * up in time, set its status word and left the device usable.  Returns RABIT_OK if so.  `status_dev`
+ * is a DEVICE word owned by the caller (4 bytes, 4-byte aligned); it holds 1 afterwards.
+ */
+RABIT_API int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us, void* stream);
+
 /* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
 RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
                  void* stream);

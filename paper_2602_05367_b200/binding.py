@@ -51,6 +51,10 @@ def _load() -> ctypes.CDLL:
     lib.rabit_linear_group.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]
     lib.rabit_linear_static_scratch.restype = _c_int
     lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
+    lib.rabit_layer_status.restype = _c_int
+    lib.rabit_layer_status.argtypes = [_c_void_p, _c_int, _c_void_p]
+    lib.rabit_selftest_bounded_wait.restype = _c_int
+    lib.rabit_selftest_bounded_wait.argtypes = [_c_void_p, _c_int, _c_void_p]
     lib.rabit_unpack.restype = _c_int
     lib.rabit_unpack.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p]
     for name in ("rabit_layer_K", "rabit_layer_M", "rabit_layer_N"):
@@ -144,6 +148,10 @@ class RabitLayer:
 
     def set_variant(self, variant: int) -> None:
         _check(_lib.rabit_set_variant(self.handle, variant))
+
+    def status(self, clear: bool = False, stream: int = 0) -> int:
+        """0 if every kernel of this layer completed its waits, RABIT_DEVICE_FAULT (-5) otherwise; synchronises."""
+        return int(_lib.rabit_layer_status(self.handle, 1 if clear else 0, _c_void_p(stream)))
 
     def unpack(self, stream: int = 0):
         planes = np.empty((self.K, self.M, self.N // 32), dtype=np.uint32)

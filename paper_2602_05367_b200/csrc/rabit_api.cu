@@ -259,6 +259,23 @@ extern "C" int rabit_linear_host(const rabit_layer* layer, const void* x_host, v
     return RABIT_OK;
 }
 
+extern "C" int rabit_layer_status(const rabit_layer* layer, int clear, void* stream) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_layer_status: layer is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned int word = 0;
+    RABIT_CUDA_TRY(cudaMemcpyAsync(&word, layer->d_status, 4, cudaMemcpyDeviceToHost, st));
+    RABIT_CUDA_TRY(cudaStreamSynchronize(st));
+    if (word != 0) {
+        if (clear) {
+            RABIT_CUDA_TRY(cudaMemsetAsync(layer->d_status, 0, 4, st));
+            RABIT_CUDA_TRY(cudaStreamSynchronize(st));
+        }
+        return rabit_fail(RABIT_DEVICE_FAULT, "rabit_layer_status: a kernel of this layer gave up on a bounded wait; its outputs are invalid");
+    }
+    return RABIT_OK;
+}
+
 extern "C" int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out, void* stream) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack: layer is NULL");

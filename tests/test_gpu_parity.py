@@ -162,3 +162,31 @@ def test_host_buffer_entry_point(batch):
     torch.cuda.synchronize()
     check_against_oracle(L, xn, yh.numpy())
     layer.free()
+
+
+def test_status_word_stays_clear_and_bounded_wait_self_test():
+    """Failure detection without a fault: after normal runs the layer's status word is clear; a kernel whose
+    wait can never succeed gives up after its limit, records it and leaves the device usable."""
+    import time
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from paper_2602_05367_b200 import binding
+    L = make_layer(300, 640, 2, key=(79,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    for batch in (1, 4, 40):
+        xn = make_x(batch, 640, key=(79, batch))
+        y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
+        assert layer.status() == 0
+        check_against_oracle(L, xn, y.cpu().numpy())
+    lib = binding.raw_lib()
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.time()
+    assert lib.rabit_selftest_bounded_wait(ctypes.c_void_p(word.data_ptr()), 20000, None) == 0, rabit.last_error()
+    assert time.time() - t0 < 5.0 and int(word.item()) == 1
+    assert lib.rabit_selftest_bounded_wait(ctypes.c_void_p(word.data_ptr()), 0, None) == -1
+    # the context is still usable
+    xn = make_x(1, 640, key=(79, 99))
+    y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
+    torch.cuda.synchronize()
+    check_against_oracle(L, xn, y.cpu().numpy())
+    layer.free()
