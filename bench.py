@@ -261,8 +261,13 @@ def bench_rabit(args) -> dict:
         def e2e_step(s):
             c = s % copies
             with torch.cuda.stream(stream):
-                for p, sh in enumerate(shapes):
-                    rabit.rabit_linear_host(layers[c][p], pin_x[sh.N][c % tokens], pin_y[p], stream=stream.cuda_stream)
+                if grouped:
+                    for grp in GROUPS:
+                        rabit.rabit_linear_group_host([layers[c][p] for p in grp], [pin_x[shapes[p].N][c % tokens] for p in grp],
+                                                      [pin_y[p] for p in grp], stream=stream.cuda_stream)
+                else:
+                    for p, sh in enumerate(shapes):
+                        rabit.rabit_linear_host(layers[c][p], pin_x[sh.N][c % tokens], pin_y[p], stream=stream.cuda_stream)
                 stream.synchronize()                  # the caller reads y on the host after every step
         for s in range(min(3 * copies, 100)):
             e2e_step(s)
@@ -277,10 +282,10 @@ def bench_rabit(args) -> dict:
         barrier()
         e_ms = max_over_ranks(ev0.elapsed_time(ev1), dist, device)
         e2e = {"value": whole_job_us_per_layer(e_ms / e2e_steps, n_proj, world), "unit": UNIT,
-               "h2d_bytes_per_step": int(sum(2 * batch * sh.N for sh in shapes)),
+               "h2d_bytes_per_step": int(sum(2 * batch * shapes[grp[0]].N for grp in GROUPS) if grouped else sum(2 * batch * sh.N for sh in shapes)),
                "d2h_bytes_per_step": int(sum(2 * batch * sh.M for sh in shapes)),
-               "steps": e2e_steps, "note": "rabit_linear_host per projection: pinned host x -> device, kernel, "
-                                           "y -> pinned host, host synchronises after every step"}
+               "steps": e2e_steps, "note": ("rabit_linear_group_host per group of projections (a shared input is copied once)" if grouped else
+                        "rabit_linear_host per projection") + ": pinned host x -> device, kernel, y -> pinned host, host synchronises after every step"}
 
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):

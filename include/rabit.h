@@ -189,6 +189,17 @@ RABIT_API int rabit_layer_status(const rabit_layer* layer, int clear, void* stre
  */
 RABIT_API int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us, void* stream);
 
+/*
+ * Host-buffer form of rabit_linear_group: inputs and outputs live in HOST memory (pinned memory makes the
+ * copies asynchronous).  An input pointer that occurs several times in xs_host is copied to the device once.
+ *   dev_stage  DEVICE, 256-byte aligned, at least rabit_group_stage_bytes(layers, n_layers, batch)
+ * Enqueues the input copies, one grouped launch and the output copies on `stream`; returns without
+ * synchronising.
+ */
+RABIT_API size_t rabit_group_stage_bytes(const rabit_layer* const* layers, int n_layers, int batch);
+RABIT_API int rabit_linear_group_host(const rabit_layer* const* layers, const void* const* xs_host, void* const* ys_host,
+                            int n_layers, int batch, void* dev_stage, size_t dev_stage_bytes, void* stream);
+
 /* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
 RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
                  void* stream);

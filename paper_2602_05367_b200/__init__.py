@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     rabit_derive_pack,
     rabit_linear,
     rabit_linear_group,
+    rabit_linear_group_host,
     rabit_linear_host,
     rabit_linear_static_scratch,
     rabit_free,

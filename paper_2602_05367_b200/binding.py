@@ -51,6 +51,10 @@ def _load() -> ctypes.CDLL:
     lib.rabit_linear_group.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]
     lib.rabit_linear_static_scratch.restype = _c_int
     lib.rabit_linear_static_scratch.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]
+    lib.rabit_group_stage_bytes.restype = _c_size_t
+    lib.rabit_group_stage_bytes.argtypes = [_c_void_p, _c_int, _c_int]
+    lib.rabit_linear_group_host.restype = _c_int
+    lib.rabit_linear_group_host.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p, _c_size_t, _c_void_p]
     lib.rabit_layer_status.restype = _c_int
     lib.rabit_layer_status.argtypes = [_c_void_p, _c_int, _c_void_p]
     lib.rabit_selftest_bounded_wait.restype = _c_int
@@ -256,6 +260,32 @@ def rabit_linear_group(layers, xs, ys, stream: Optional[int] = None):
     yp = (_c_void_p * n)(*[y.data_ptr() for y in ys])
     _check(_lib.rabit_linear_group(h, xp, yp, n, batch, _c_void_p(st)))
     return ys
+
+
+def rabit_linear_group_host(layers, xs_host, ys_host, stream: Optional[int] = None):
+    """Host-buffer form of rabit_linear_group: CPU float16 tensors in and out (pinned for asynchronous copies);
+    an input tensor that occurs several times is copied once.  Returns without synchronising."""
+    import torch
+
+    n = len(layers)
+    if n < 1 or len(xs_host) != n or len(ys_host) != n:
+        raise ValueError("layers, xs_host and ys_host must have the same, non-zero length")
+    batch = 1 if xs_host[0].dim() == 1 else xs_host[0].shape[0]
+    for L, x, y in zip(layers, xs_host, ys_host):
+        if x.dtype != torch.float16 or x.is_cuda or not x.is_contiguous() or x.numel() != batch * L.N:
+            raise ValueError("every x must be a contiguous CPU float16 tensor of batch*N elements")
+        if y.dtype != torch.float16 or y.is_cuda or not y.is_contiguous() or y.numel() != batch * L.M:
+            raise ValueError("every y must be a contiguous CPU float16 tensor of batch*M elements")
+    h = (_c_void_p * n)(*[L.handle for L in layers])
+    need = int(_lib.rabit_group_stage_bytes(h, n, batch))
+    first = layers[0]
+    if first._stage is None or first._stage.numel() < need:
+        first._stage = torch.empty(need, dtype=torch.uint8, device=first.dev_buf.device)
+    st = torch.cuda.current_stream(first.dev_buf.device).cuda_stream if stream is None else stream
+    xp = (_c_void_p * n)(*[x.data_ptr() for x in xs_host])
+    yp = (_c_void_p * n)(*[y.data_ptr() for y in ys_host])
+    _check(_lib.rabit_linear_group_host(h, xp, yp, n, batch, _c_void_p(first._stage.data_ptr()), need, _c_void_p(st)))
+    return ys_host
 
 
 def rabit_linear_host(layer: RabitLayer, x_host, y_host, stream: Optional[int] = None):

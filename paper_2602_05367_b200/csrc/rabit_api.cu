@@ -259,6 +259,54 @@ extern "C" int rabit_linear_host(const rabit_layer* layer, const void* x_host, v
     return RABIT_OK;
 }
 
+extern "C" size_t rabit_group_stage_bytes(const rabit_layer* const* layers, int n_layers, int batch) {
+    if (!layers || n_layers < 1 || n_layers > 8 || batch < 1) return 0;
+    size_t total = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!layers[l]) return 0;
+        total += rabit_align256((size_t)batch * layers[l]->geom.N * 2) + rabit_align256((size_t)batch * layers[l]->geom.M * 2);
+    }
+    return total;
+}
+
+extern "C" int rabit_linear_group_host(const rabit_layer* const* layers, const void* const* xs_host, void* const* ys_host,
+                                       int n_layers, int batch, void* dev_stage, size_t dev_stage_bytes, void* stream) {
+    rabit_clear_error();
+    if (!layers || !xs_host || !ys_host || !dev_stage) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group_host: null pointer");
+    if (n_layers < 1 || n_layers > 8) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group_host: n_layers must be 1..8 (got %d)", n_layers);
+    if (batch < 1) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group_host: batch must be >= 1 (got %d)", batch);
+    if (((uintptr_t)dev_stage & 255u) != 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group_host: dev_stage must be 256-byte aligned");
+    for (int l = 0; l < n_layers; ++l)
+        if (!layers[l] || !xs_host[l] || !ys_host[l]) return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group_host: null entry %d", l);
+    const size_t need = rabit_group_stage_bytes(layers, n_layers, batch);
+    if (dev_stage_bytes < need)
+        return rabit_fail(RABIT_BUFFER_TOO_SMALL, "rabit_linear_group_host: stage holds %zu bytes, need %zu", dev_stage_bytes, need);
+    cudaStream_t st = (cudaStream_t)stream;
+    char* cur = (char*)dev_stage;
+    const void* dx[8];
+    void* dy[8];
+    for (int l = 0; l < n_layers; ++l) {
+        const size_t xb = (size_t)batch * layers[l]->geom.N * 2;
+        dx[l] = nullptr;
+        for (int m = 0; m < l; ++m)                                      // the same host input (and width) again: reuse its copy
+            if (xs_host[m] == xs_host[l] && layers[m]->geom.N == layers[l]->geom.N) { dx[l] = dx[m]; break; }
+        if (!dx[l]) {
+            RABIT_CUDA_TRY(cudaMemcpyAsync(cur, xs_host[l], xb, cudaMemcpyHostToDevice, st));
+            dx[l] = cur;
+            cur += rabit_align256(xb);
+        }
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        dy[l] = cur;
+        cur += rabit_align256((size_t)batch * layers[l]->geom.M * 2);
+    }
+    int rc = rabit_linear_group(layers, dx, dy, n_layers, batch, stream);
+    if (rc != RABIT_OK) return rc;
+    for (int l = 0; l < n_layers; ++l)
+        RABIT_CUDA_TRY(cudaMemcpyAsync(ys_host[l], dy[l], (size_t)batch * layers[l]->geom.M * 2, cudaMemcpyDeviceToHost, st));
+    return RABIT_OK;
+}
+
 extern "C" int rabit_layer_status(const rabit_layer* layer, int clear, void* stream) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_layer_status: layer is NULL");

@@ -73,3 +73,22 @@ def test_group_falls_back_for_large_batch_and_checks_arguments():
     assert lib.rabit_linear_group(h, xp, yp, 0, 1, None) == -1
     assert lib.rabit_linear_group(None, xp, yp, 1, 1, None) == -1
     layer.free()
+
+
+def test_group_host_buffers():
+    """rabit_linear_group_host: pinned host inputs (one shared by two layers) and outputs."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    specs = [(2, 300, 640), (2, 128, 640), (3, 200, 96)]
+    Ls = [make_layer(M, N, K, key=(44, i)) for i, (K, M, N) in enumerate(specs)]
+    layers = [rabit.rabit_pack(L.planes, L.g, L.h) for L in Ls]
+    for batch in (1, 3):
+        xa = make_x(batch, 640, key=(44, batch, 1)); xb = make_x(batch, 96, key=(44, batch, 2))
+        pa, pb = torch.from_numpy(xa).pin_memory(), torch.from_numpy(xb).pin_memory()
+        ys = [torch.zeros((batch, L.M), dtype=torch.float16).pin_memory() for L in Ls]
+        rabit.rabit_linear_group_host(layers, [pa, pa, pb], ys)
+        torch.cuda.synchronize()
+        for L, a, y in zip(Ls, [xa, xa, xb], ys):
+            check_against_oracle(L, a, y.numpy())
+    for layer in layers:
+        layer.free()
