@@ -89,20 +89,19 @@ struct GemvParams {
     __half* y;
     float* partial;          // [n_rt*K + grid][RABIT_PARTIAL_BATCH][128]
                              // segment (CTA c, strip s) uses slot c + s; every word rests at kSentinel between calls
-    int n_tiles;             // n_rt * K * n_ct
-    int base;                // position of this layer's first tile in the launch's tile numbering
-    FastDiv div_c, div_k, div_kc;   // by n_ct, K, K * n_ct
+    int n_tiles;             // n_rt * K * n_ct (< 2^31)
+    int cta0, n_cta;         // the CTAs blockIdx.x = cta0 .. cta0 + n_cta - 1 work on this layer
+    int q, r;                // n_tiles = q * n_cta + r: the layer's CTAs 0..r-1 own q+1 tiles, the others q
+    FastDiv div_c, div_k, div_kc, div_q, div_q1;   // by n_ct, K, K * n_ct, q, q + 1
 };
 
 // A launch runs up to kMaxGroup layers that do not depend on one another (for example the
-// projections that read the same activations); their tiles are numbered one layer after the
-// other and that whole range is split evenly over the CTAs.
+// projections that read the same activations).  The CTAs of the grid are shared out among the
+// layers in proportion to their tiles, so every CTA works on exactly one layer and the tiles of
+// a layer are split evenly over its CTAs.
 constexpr int kMaxGroup = 8;
 struct GroupParams {
     int n_layers;
-    int total_tiles;         // < 2^31
-    int q, r;                // total_tiles = q * grid + r: CTAs 0..r-1 own q+1 tiles, the others q
-    FastDiv div_q, div_q1;   // by q, q + 1
     unsigned int* status;
     int nb;                  // batch rows actually present (<= the kernel's NB); the others are neither read nor written
     GemvParams layer[kMaxGroup];
@@ -164,9 +163,10 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 
 // Even split of the tile positions: CTA c owns [c*q + min(c, r), (c+1)*q + min(c+1, r)).
 __device__ __forceinline__ int range_lo(int c, int q, int r) { return c * q + min(c, r); }
-__device__ __forceinline__ int cta_of(int p, const GroupParams& GP) {
-    const int big = GP.r * (GP.q + 1);           // positions owned by the CTAs that have q+1 tiles
-    return p < big ? fdiv(p, GP.div_q1) : GP.r + fdiv(p - big, GP.div_q);
+// The CTA (counted inside its layer) that owns tile position p of that layer.
+__device__ __forceinline__ int cta_of(int p, const GemvParams& P) {
+    const int big = P.r * (P.q + 1);             // positions owned by the CTAs that have q+1 tiles
+    return p < big ? fdiv(p, P.div_q1) : P.r + fdiv(p - big, P.div_q);
 }
 
 // sigma = 2^s with |h x| * sigma < 2^28 for every column; inv = 2^-s (NaN if the inputs are not finite).
@@ -239,8 +239,6 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     Smem<NB>& S = *reinterpret_cast<Smem<NB>*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nb = GP.nb;
-    const int glo = range_lo(blockIdx.x, GP.q, GP.r);                      // this CTA's range in the launch's numbering
-    const int ghi = range_lo(blockIdx.x + 1, GP.q, GP.r);
     volatile int* abort_flag = &S.abort_flag;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -255,17 +253,18 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     }
     __syncthreads();
 
-    // One pass per layer that meets this CTA's range.  `it0` counts the stages of the earlier passes: the
-    // ring slots and barrier phases simply continue from pass to pass.
+    // The layer this CTA works on (the loop body runs once; it is written as passes with a running stage
+    // counter `it0`, so ring slots and barrier phases would simply continue if a CTA ever took several layers).
     int it0 = 0;
     bool first_pass = true;
     for (int li = 0; li < GP.n_layers; ++li) {
     const GemvParams& P = GP.layer[li];
-    if (P.base + P.n_tiles <= glo || P.base >= ghi) continue;
+    if ((int)blockIdx.x < P.cta0 || (int)blockIdx.x >= P.cta0 + P.n_cta) continue;
     const RabitGeom& G = P.G;
     const int C = G.n_ct;
-    const int lo = max(glo, P.base) - P.base;                              // this pass's range, in the layer's own numbering
-    const int n_tiles = min(ghi, P.base + P.n_tiles) - P.base - lo;
+    const int me = (int)blockIdx.x - P.cta0;                               // this CTA's index among the layer's CTAs
+    const int lo = range_lo(me, P.q, P.r);                                 // its tile range, in the layer's own numbering
+    const int n_tiles = range_lo(me + 1, P.q, P.r) - lo;
     const int n_stages = (n_tiles + kStageTiles - 1) / kStageTiles;
     if (!first_pass) {                                                     // every warp is done with the previous pass
         __syncthreads();
@@ -450,7 +449,6 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
             for (int c = 0; c < 4; ++c) acc[jp][p][c] = 0;
 #pragma unroll
     for (int b = 0; b < NB; ++b) sum_t[b] = 0;
-    const int me = blockIdx.x;
     const int KC = G.K * C;
     bool red_in_use = false;
 
@@ -595,7 +593,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
 #pragma unroll 1
                 for (int kk = 0; kk < G.K; ++kk) {
                     const int s0 = (rt_f * G.K + kk) * C;
-                    const int c0 = cta_of(P.base + s0, GP), c1 = cta_of(P.base + s0 + C - 1, GP);
+                    const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
                     unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
                                         (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + b) * RABIT_TILE_ROWS + red_r;
 #pragma unroll 1
@@ -691,9 +689,9 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
     if (batch < 1 || batch > 4) return cudaErrorInvalidValue;
     GroupParams GP;
     GP.n_layers = n_layers;
-    GP.total_tiles = 0;
     GP.status = layers[0]->d_status;
     GP.nb = batch;
+    long long total = 0;
     for (int l = 0; l < n_layers; ++l) {
         const rabit_layer& L = *layers[l];
         GemvParams& P = GP.layer[l];
@@ -705,24 +703,57 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
         P.y = (__half*)ys[l];
         P.partial = L.d_partial;
         P.n_tiles = L.geom.n_rt * L.geom.K * L.geom.n_ct;
-        P.base = GP.total_tiles;
         P.div_c = make_fastdiv((unsigned int)L.geom.n_ct);
         P.div_k = make_fastdiv((unsigned int)L.geom.K);
         P.div_kc = make_fastdiv((unsigned int)(L.geom.K * L.geom.n_ct));
-        GP.total_tiles += P.n_tiles;
+        total += P.n_tiles;
     }
-    for (int l = n_layers; l < kMaxGroup; ++l) GP.layer[l] = GP.layer[0];
     const int sms = layers[0]->sm_count > 0 ? layers[0]->sm_count : 148;
-    int grid = (batch <= 2 ? 2 : 1) * sms;                   // as many CTAs as are resident at once (two per SM up to two batch rows)
-    if (grid > RABIT_MAX_GRID) grid = RABIT_MAX_GRID;
-    if (grid > GP.total_tiles) grid = GP.total_tiles;
-    GP.q = GP.total_tiles / grid;
-    GP.r = GP.total_tiles % grid;
-    GP.div_q = make_fastdiv((unsigned int)GP.q);
-    GP.div_q1 = make_fastdiv((unsigned int)GP.q + 1u);
-    if (batch == 1) return launch_nb<1>(GP, grid, stream);
-    if (batch == 2) return launch_nb<2>(GP, grid, stream);
-    return launch_nb<4>(GP, grid, stream);
+    long long grid_ll = (long long)(batch <= 2 ? 2 : 1) * sms;   // as many CTAs as are resident at once (two per SM up to two batch rows)
+    if (grid_ll > RABIT_MAX_GRID) grid_ll = RABIT_MAX_GRID;
+    if (grid_ll > total) grid_ll = total;
+    if (grid_ll < n_layers) grid_ll = n_layers;
+    const int grid = (int)grid_ll;
+    // share the CTAs out in proportion to the tiles: floor first (at least one each, at most one per tile),
+    // then hand the rest to the layers with the most tiles per CTA
+    int given = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        GemvParams& P = GP.layer[l];
+        long long n = (long long)grid * P.n_tiles / total;
+        if (n < 1) n = 1;
+        if (n > P.n_tiles) n = P.n_tiles;
+        P.n_cta = (int)n;
+        given += P.n_cta;
+    }
+    while (given > grid) {                                   // the "at least one" floor can overshoot: take from the best-served layer
+        int best = -1;
+        for (int l = 0; l < n_layers; ++l)
+            if (GP.layer[l].n_cta > 1 && (best < 0 || (long long)GP.layer[l].n_tiles * GP.layer[best].n_cta < (long long)GP.layer[best].n_tiles * GP.layer[l].n_cta)) best = l;
+        if (best < 0) break;
+        GP.layer[best].n_cta -= 1; given -= 1;
+    }
+    while (given < grid) {
+        int best = -1;
+        for (int l = 0; l < n_layers; ++l)
+            if (GP.layer[l].n_cta < GP.layer[l].n_tiles && (best < 0 || (long long)GP.layer[l].n_tiles * GP.layer[best].n_cta > (long long)GP.layer[best].n_tiles * GP.layer[l].n_cta)) best = l;
+        if (best < 0) break;
+        GP.layer[best].n_cta += 1; given += 1;
+    }
+    int c0 = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        GemvParams& P = GP.layer[l];
+        P.cta0 = c0;
+        c0 += P.n_cta;
+        P.q = P.n_tiles / P.n_cta;
+        P.r = P.n_tiles % P.n_cta;
+        P.div_q = make_fastdiv((unsigned int)P.q);
+        P.div_q1 = make_fastdiv((unsigned int)P.q + 1u);
+    }
+    for (int l = n_layers; l < kMaxGroup; ++l) { GP.layer[l] = GP.layer[0]; GP.layer[l].n_cta = 0; }
+    const int launch_grid = c0;
+    if (batch == 1) return launch_nb<1>(GP, launch_grid, stream);
+    if (batch == 2) return launch_nb<2>(GP, launch_grid, stream);
+    return launch_nb<4>(GP, launch_grid, stream);
 }
 
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
