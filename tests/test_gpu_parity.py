@@ -190,3 +190,42 @@ def test_status_word_stays_clear_and_bounded_wait_self_test():
     torch.cuda.synchronize()
     check_against_oracle(L, xn, y.cpu().numpy())
     layer.free()
+
+
+@pytest.mark.parametrize("batch", [2, 4, 40])
+def test_non_finite_activations_poison_only_their_batch_row(batch):
+    """An inf or NaN in one activation row makes every output of that row non-finite and leaves the other
+    rows within tolerance (GEMV: the fixed-point scale of the row becomes NaN; GEMM: inf/NaN propagate)."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(300, 640, 2, key=(66, batch))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    xn = make_x(batch, 640, key=(66, batch))
+    bad = xn.copy()
+    bad[1, 17] = np.float16(np.inf)
+    y = rabit.rabit_linear(layer, torch.from_numpy(bad).cuda()).cpu().numpy().astype(np.float64)
+    assert not np.isfinite(y[1]).any()
+    keep = [b for b in range(batch) if b != 1]
+    ref = orc.linear(L.planes, L.g, L.h, xn[keep])
+    tol = orc.tolerance(L.g, L.h, xn[keep])
+    assert (np.abs(y[keep] - ref).max(axis=1) <= tol).all()
+    bad[1, 17] = np.float16(np.nan)
+    y = rabit.rabit_linear(layer, torch.from_numpy(bad).cuda()).cpu().numpy()
+    assert np.isnan(y[1].astype(np.float64)).all()
+    assert layer.status() == 0
+    layer.free()
+
+
+def test_tiny_and_huge_magnitudes_keep_their_precision():
+    """The fixed-point scale follows the data: activations of magnitude 1e-4 or 1e+4 lose nothing."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(256, 1024, 2, key=(67,))
+    layer = rabit.rabit_pack(L.planes, L.g, L.h)
+    for scale in (1e-4, 1.0, 3e3):
+        xn = (make_x(2, 1024, key=(67,)).astype(np.float32) * scale).astype(np.float16)
+        y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
+        torch.cuda.synchronize()
+        err, tol = check_against_oracle(L, xn, y.cpu().numpy())
+        assert (err <= 0.3 * tol).all()          # far inside: only the fp16 output rounding is left
+    layer.free()
