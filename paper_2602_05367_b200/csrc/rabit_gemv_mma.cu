@@ -579,50 +579,76 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
         next_segment();
     }
 
-    // ---- finish the row tiles whose last tile this CTA owns.  Every reducer thread works alone on its
-    //      (batch row, row) words: it reads that word of every contributor's partial, path by path and CTA
-    //      by CTA, waits (bounded) while a word still holds the sentinel, restores the sentinel for the next
-    //      call, adds in that fixed order and stores fp16.  No barrier and no fence is involved: a partial
+    // ---- finish the row tiles whose last tile this CTA owns.  The two halves of the MMA threads share the
+    //      paths (half = path & 1).  Thread (half, r) reads row r's word of every contributor's partial of its
+    //      paths, for all batch rows at once (up to 8 contributors x NB words in flight), waits (bounded) while a
+    //      word still holds the sentinel, restores the sentinel for the next call and adds in that fixed order.
+    //      The halves meet in shared memory and the first one stores fp16.  No fence is involved: a partial
     //      word carries no other data with it.
-    if (reducer) {
+    {
         constexpr size_t kStride = (size_t)RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS;
+        constexpr int kFan = 8;
+        const int half = (tid >> 7) & 1;
+        const bool two_halves = G.K > 1;
         for (int rt_f = fdiv(lo, P.div_kc); (rt_f + 1) * KC - 1 < lo + n_tiles; ++rt_f) {
-#pragma unroll 1
-            for (int b = red_b0; b < nb; b += 2) {
-                float sum = 0.f;
-#pragma unroll 1
-                for (int kk = 0; kk < G.K; ++kk) {
-                    const int s0 = (rt_f * G.K + kk) * C;
-                    const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
-                    unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
-                                        (((size_t)c0 + (size_t)rt_f * G.K + kk) * RABIT_PARTIAL_BATCH + b) * RABIT_TILE_ROWS + red_r;
-#pragma unroll 1
-                    for (int c = c0; c <= c1; c += 8) {                        // eight loads in flight, consumed in order
-                        unsigned int v[8];
+            float part[NB];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            v[u] = 0u;
-                            if (c + u <= c1) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
+            for (int b = 0; b < NB; ++b) part[b] = 0.f;
+#pragma unroll 1
+            for (int kk = half; kk < G.K; kk += 2) {
+                const int s0 = (rt_f * G.K + kk) * C;
+                const int c0 = cta_of(s0, P), c1 = cta_of(s0 + C - 1, P);
+                unsigned int* src = reinterpret_cast<unsigned int*>(P.partial) +
+                                    ((size_t)c0 + (size_t)rt_f * G.K + kk) * kStride + red_r;
+#pragma unroll 1
+                for (int c = c0; c <= c1; c += kFan) {
+                    unsigned int v[NB][kFan];
+#pragma unroll
+                    for (int b = 0; b < NB; ++b)
+#pragma unroll
+                        for (int u = 0; u < kFan; ++u) {
+                            v[b][u] = 0u;
+                            if (b < nb && c + u <= c1)
+                                asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[b][u]) : "l"(src + u * kStride + b * RABIT_TILE_ROWS) : "memory");
                         }
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            if (c + u > c1) break;
-                            if (v[u] == kSentinel) {
+                    for (int u = 0; u < kFan; ++u) {
+                        if (c + u > c1) break;
+#pragma unroll
+                        for (int b = 0; b < NB; ++b) {
+                            if (b >= nb) break;
+                            unsigned int* word = src + u * kStride + b * RABIT_TILE_ROWS;
+                            if (v[b][u] == kSentinel) {
                                 const long long t0 = clock64();
                                 do {
-                                    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[u]) : "l"(src + u * kStride) : "memory");
-                                    if (v[u] != kSentinel) break;
+                                    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[b][u]) : "l"(word) : "memory");
+                                    if (v[b][u] != kSentinel) break;
                                     if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
                                 } while (true);
                             }
-                            __stcg(src + u * kStride, kSentinel);
-                            sum += __uint_as_float(v[u]);
+                            __stcg(word, kSentinel);
+                            part[b] += __uint_as_float(v[b][u]);
                         }
-                        src += 8 * kStride;
                     }
+                    src += kFan * kStride;
                 }
+            }
+            if (two_halves) {
+                bar_mma_warps();                                               // the last flush's readers are done with S.red
+                if (half) {
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) S.red[0][b][red_r] = part[b];
+                }
+                bar_mma_warps();
+            }
+            if (!half) {
                 const int row = rt_f * RABIT_TILE_ROWS + red_r;
-                if (row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(sum);
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (b >= nb) break;
+                    const float sum = two_halves ? part[b] + S.red[0][b][red_r] : part[b];
+                    if (row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(sum);
+                }
             }
         }
     }
