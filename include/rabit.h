@@ -138,7 +138,10 @@ RABIT_API int rabit_linear_group(const rabit_layer* const* layers, const void* c
  *   y_host  HOST fp16 [batch][M]
  *   dev_stage DEVICE, 256-byte aligned, caller-owned, at least rabit_stage_bytes(layer, batch)
  * Enqueues on `stream`: copy x to the stage, the layer kernel, copy y back.  Returns without
- * synchronising; y_host is valid once the stream has reached this point.
+ * synchronising; y_host is valid once the stream has reached this point.  If y_host is page-locked,
+ * mapped memory (cudaHostAlloc / cudaHostRegister, 16-byte aligned) and batch <= 16, the kernel stores
+ * its result there itself and no copy back is enqueued; y_host must then not be read before the stream
+ * has reached this point either.
  */
 RABIT_API size_t rabit_stage_bytes(const rabit_layer* layer, int batch);
 RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, void* y_host, int batch,
@@ -194,7 +197,8 @@ RABIT_API int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us
  * copies asynchronous).  An input pointer that occurs several times in xs_host is copied to the device once.
  *   dev_stage  DEVICE, 256-byte aligned, at least rabit_group_stage_bytes(layers, n_layers, batch)
  * Enqueues the input copies, one grouped launch and the output copies on `stream`; returns without
- * synchronising.
+ * synchronising.  Outputs in page-locked, mapped host memory are written by the kernel itself when
+ * batch <= 16 (see rabit_linear_host).
  */
 RABIT_API size_t rabit_group_stage_bytes(const rabit_layer* const* layers, int n_layers, int batch);
 RABIT_API int rabit_linear_group_host(const rabit_layer* const* layers, const void* const* xs_host, void* const* ys_host,

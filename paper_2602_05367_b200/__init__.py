@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     rabit_linear,
     rabit_linear_group,
     rabit_linear_group_host,
+    PreparedGroupHost,
     rabit_linear_host,
     rabit_linear_static_scratch,
     rabit_free,

@@ -288,6 +288,44 @@ def rabit_linear_group_host(layers, xs_host, ys_host, stream: Optional[int] = No
     return ys_host
 
 
+class PreparedGroupHost:
+    """A rabit_linear_group_host call with its arguments checked and marshalled once: calling the object enqueues
+    the same copies and launch again on the given stream (the tensors are kept alive and read / written in place),
+    without the per-call checks of rabit_linear_group_host.  Returns without synchronising."""
+
+    def __init__(self, layers, xs_host, ys_host):
+        import torch
+
+        n = len(layers)
+        if n < 1 or len(xs_host) != n or len(ys_host) != n:
+            raise ValueError("layers, xs_host and ys_host must have the same, non-zero length")
+        batch = 1 if xs_host[0].dim() == 1 else xs_host[0].shape[0]
+        for L, x, y in zip(layers, xs_host, ys_host):
+            if x.dtype != torch.float16 or x.is_cuda or not x.is_contiguous() or x.numel() != batch * L.N:
+                raise ValueError("every x must be a contiguous CPU float16 tensor of batch*N elements")
+            if y.dtype != torch.float16 or y.is_cuda or not y.is_contiguous() or y.numel() != batch * L.M:
+                raise ValueError("every y must be a contiguous CPU float16 tensor of batch*M elements")
+        self._keep = (list(layers), list(xs_host), list(ys_host))
+        self._device = layers[0].dev_buf.device
+        self._h = (_c_void_p * n)(*[L.handle for L in layers])
+        self._xp = (_c_void_p * n)(*[x.data_ptr() for x in xs_host])
+        self._yp = (_c_void_p * n)(*[y.data_ptr() for y in ys_host])
+        self._n, self._batch = n, batch
+        self._need = int(_lib.rabit_group_stage_bytes(self._h, n, batch))
+        self._stage = torch.empty(self._need, dtype=torch.uint8, device=self._device)
+        self._stage_ptr = _c_void_p(self._stage.data_ptr())
+        self.ys_host = ys_host
+
+    def __call__(self, stream: Optional[int] = None):
+        if stream is None:
+            import torch
+            stream = torch.cuda.current_stream(self._device).cuda_stream
+        rc = _lib.rabit_linear_group_host(self._h, self._xp, self._yp, self._n, self._batch, self._stage_ptr, self._need, _c_void_p(stream))
+        if rc != 0:
+            _check(rc)
+        return self.ys_host
+
+
 def rabit_linear_host(layer: RabitLayer, x_host, y_host, stream: Optional[int] = None):
     """Host-buffer form: x_host / y_host are CPU float16 tensors (pinned for asynchronous copies)
     of shape [batch][N] (or [N]) and [batch][M]; the copies and the kernel are enqueued on the

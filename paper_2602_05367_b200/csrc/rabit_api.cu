@@ -238,6 +238,20 @@ extern "C" size_t rabit_stage_bytes(const rabit_layer* layer, int batch) {
     return rabit_align256((size_t)batch * layer->geom.N * 2) + rabit_align256((size_t)batch * layer->geom.M * 2);
 }
 
+// Device address under which the GPU can store straight into a host buffer of `bytes` bytes (page-locked,
+// mapped memory, 16-byte aligned), or nullptr if the buffer is ordinary pageable memory.
+static void* mapped_output_alias(void* host_ptr, size_t bytes) {
+    cudaPointerAttributes first, last;
+    if (cudaPointerGetAttributes(&first, host_ptr) != cudaSuccess || cudaPointerGetAttributes(&last, (char*)host_ptr + bytes - 1) != cudaSuccess) {
+        cudaGetLastError();                                              // not an error of the caller: fall back to a copy
+        return nullptr;
+    }
+    if (first.type != cudaMemoryTypeHost || last.type != cudaMemoryTypeHost || !first.devicePointer || !last.devicePointer) return nullptr;
+    if ((char*)last.devicePointer - (char*)first.devicePointer != (ptrdiff_t)(bytes - 1)) return nullptr;
+    if (((uintptr_t)first.devicePointer & 15u) != 0) return nullptr;
+    return first.devicePointer;
+}
+
 extern "C" int rabit_linear_host(const rabit_layer* layer, const void* x_host, void* y_host, int batch,
                                  void* dev_stage, size_t dev_stage_bytes, void* stream) {
     rabit_clear_error();
@@ -253,9 +267,12 @@ extern "C" int rabit_linear_host(const rabit_layer* layer, const void* x_host, v
     char* dy = dx + rabit_align256(xb);
     cudaStream_t st = (cudaStream_t)stream;
     RABIT_CUDA_TRY(cudaMemcpyAsync(dx, x_host, xb, cudaMemcpyHostToDevice, st));
-    int rc = rabit_linear(layer, dx, dy, batch, stream);
+    // A decode-sized result goes straight to mapped host memory from the kernel's last stores (a few KB; the
+    // copy engine's latency for so small a copy is longer than the kernel); anything else through the stage.
+    void* direct = batch <= RABIT_MAX_GEMV_BATCH ? mapped_output_alias(y_host, yb) : nullptr;
+    int rc = rabit_linear(layer, dx, direct ? direct : dy, batch, stream);
     if (rc != RABIT_OK) return rc;
-    RABIT_CUDA_TRY(cudaMemcpyAsync(y_host, dy, yb, cudaMemcpyDeviceToHost, st));
+    if (!direct) RABIT_CUDA_TRY(cudaMemcpyAsync(y_host, dy, yb, cudaMemcpyDeviceToHost, st));
     return RABIT_OK;
 }
 
@@ -296,14 +313,18 @@ extern "C" int rabit_linear_group_host(const rabit_layer* const* layers, const v
             cur += rabit_align256(xb);
         }
     }
-    for (int l = 0; l < n_layers; ++l) {
-        dy[l] = cur;
-        cur += rabit_align256((size_t)batch * layers[l]->geom.M * 2);
+    bool staged[8];
+    for (int l = 0; l < n_layers; ++l) {                                 // decode-sized results: straight to mapped host memory (see rabit_linear_host)
+        const size_t yb = (size_t)batch * layers[l]->geom.M * 2;
+        void* direct = batch <= RABIT_MAX_GEMV_BATCH ? mapped_output_alias(ys_host[l], yb) : nullptr;
+        staged[l] = direct == nullptr;
+        dy[l] = direct ? direct : cur;
+        cur += rabit_align256(yb);
     }
     int rc = rabit_linear_group(layers, dx, dy, n_layers, batch, stream);
     if (rc != RABIT_OK) return rc;
     for (int l = 0; l < n_layers; ++l)
-        RABIT_CUDA_TRY(cudaMemcpyAsync(ys_host[l], dy[l], (size_t)batch * layers[l]->geom.M * 2, cudaMemcpyDeviceToHost, st));
+        if (staged[l]) RABIT_CUDA_TRY(cudaMemcpyAsync(ys_host[l], dy[l], (size_t)batch * layers[l]->geom.M * 2, cudaMemcpyDeviceToHost, st));
     return RABIT_OK;
 }
 

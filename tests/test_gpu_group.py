@@ -85,10 +85,32 @@ def test_group_host_buffers():
     for batch in (1, 3):
         xa = make_x(batch, 640, key=(44, batch, 1)); xb = make_x(batch, 96, key=(44, batch, 2))
         pa, pb = torch.from_numpy(xa).pin_memory(), torch.from_numpy(xb).pin_memory()
-        ys = [torch.zeros((batch, L.M), dtype=torch.float16).pin_memory() for L in Ls]
+        ys = [torch.zeros((batch, L.M), dtype=torch.float16) for L in Ls]
+        ys = [y.pin_memory() if i != 1 else y for i, y in enumerate(ys)]     # one pageable output: staged copy back
         rabit.rabit_linear_group_host(layers, [pa, pa, pb], ys)
         torch.cuda.synchronize()
         for L, a, y in zip(Ls, [xa, xa, xb], ys):
             check_against_oracle(L, a, y.numpy())
+    for layer in layers:
+        layer.free()
+
+
+def test_prepared_group_host_call_repeats():
+    """PreparedGroupHost: marshalled once, called three times with new inputs written into the same host tensors."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    specs = [(2, 300, 640), (2, 128, 640)]
+    Ls = [make_layer(M, N, K, key=(45, i)) for i, (K, M, N) in enumerate(specs)]
+    layers = [rabit.rabit_pack(L.planes, L.g, L.h) for L in Ls]
+    px = torch.zeros((2, 640), dtype=torch.float16).pin_memory()
+    ys = [torch.zeros((2, L.M), dtype=torch.float16).pin_memory() for L in Ls]
+    call = rabit.PreparedGroupHost(layers, [px, px], ys)
+    for rep in range(3):
+        xa = make_x(2, 640, key=(45, rep))
+        px.copy_(torch.from_numpy(xa))
+        call()
+        torch.cuda.synchronize()
+        for L, y in zip(Ls, ys):
+            check_against_oracle(L, xa, y.numpy())
     for layer in layers:
         layer.free()

@@ -148,19 +148,25 @@ def test_argument_errors_on_device():
     layer.free()
 
 
-@pytest.mark.parametrize("batch", [1, 3])
-def test_host_buffer_entry_point(batch):
-    """rabit_linear_host: pinned host x in, pinned host y out, copies enqueued by the library."""
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("batch", [1, 3, 40])
+def test_host_buffer_entry_point(batch, pinned):
+    """rabit_linear_host: host x in, host y out.  Pinned (mapped) outputs of decode-sized calls are written
+    by the kernel itself, everything else goes through the device stage and a copy back; twice in a row."""
     import torch
     import paper_2602_05367_b200 as rabit
     L = make_layer(200, 640, 2, key=(78,))
     layer = rabit.rabit_pack(L.planes, L.g, L.h)
-    xn = make_x(batch, 640, key=(78, batch))
-    xh = torch.from_numpy(xn).pin_memory()
-    yh = torch.zeros((batch, 200), dtype=torch.float16).pin_memory()
-    rabit.rabit_linear_host(layer, xh, yh)
-    torch.cuda.synchronize()
-    check_against_oracle(L, xn, yh.numpy())
+    for rep in range(2):
+        xn = make_x(batch, 640, key=(78, batch, rep))
+        xh = torch.from_numpy(xn)
+        yh = torch.zeros((batch, 200), dtype=torch.float16)
+        if pinned:
+            xh, yh = xh.pin_memory(), yh.pin_memory()
+        rabit.rabit_linear_host(layer, xh, yh)
+        torch.cuda.synchronize()
+        check_against_oracle(L, xn, yh.numpy())
+    assert layer.status() == 0
     layer.free()
 
 
