@@ -186,6 +186,12 @@ __device__ __forceinline__ void choose_scale(unsigned int xmax_bits, float hmax,
 }
 
 
+// The 32 words of a tile's table row (per batch row) span all 32 banks, and the lanes of a builder warp write the
+// same few words of eight different tiles at once: unrotated that is an 8-way bank conflict on every store.  Row j
+// is therefore rotated by table_rot_pairs(j) word pairs, which spreads the eight tiles over distinct banks; a
+// reader of tile j adds the same rotation to its pair index.
+__device__ __forceinline__ int table_rot_pairs(int j) { return (j & 1) + ((j >> 1) & 3) * 4; }
+
 // One lane's share of a stage: columns 8*bv .. +7 of tile j for ROWS batch rows starting at b0
 // -> digit words in fragment order + the sum of T over those columns.
 template <int NB, int ROWS>
@@ -208,6 +214,7 @@ __device__ __forceinline__ void build_rows(Smem<NB>& S, int slot, int j, int bv,
 #pragma unroll
         for (int c = 0; c < 8; ++c) tsum += Tq[c];
         uint32_t* tbl = reinterpret_cast<uint32_t*>(&S.table[slot][j][(b0 + rr) * 16]);
+        const int rot = table_rot_pairs(j) * 2;
 #pragma unroll
         for (int hlf = 0; hlf < 2; ++hlf) {  // columns 8*bv + 4*hlf .. +3  <->  group u = 2*bv + hlf
             const int u = 2 * bv + hlf;
@@ -216,11 +223,11 @@ __device__ __forceinline__ void build_rows(Smem<NB>& S, int slot, int j, int bv,
             for (int c = 0; c < 4; ++c) X[c] = ((uint32_t)Tq[4 * hlf + c] + 0x80808080u) ^ 0x80808080u;   // bytes = balanced digits
             const uint32_t t0 = __byte_perm(X[0], X[1], 0x5140), t1 = __byte_perm(X[2], X[3], 0x5140);
             const uint32_t t2 = __byte_perm(X[0], X[1], 0x7362), t3 = __byte_perm(X[2], X[3], 0x7362);
-            uint32_t* dst = tbl + (u & 3) * 2 + (u >> 2);
-            dst[0] = __byte_perm(t0, t1, 0x5410);                     // word pair index 4*digit + tq
-            dst[8] = __byte_perm(t0, t1, 0x7632);
-            dst[16] = __byte_perm(t2, t3, 0x5410);
-            dst[24] = __byte_perm(t2, t3, 0x7632);
+            const int at = (u & 3) * 2 + (u >> 2) + rot;              // word pair index 4*digit + tq, rotated by the tile's offset
+            tbl[at & 31] = __byte_perm(t0, t1, 0x5410);
+            tbl[(at + 8) & 31] = __byte_perm(t0, t1, 0x7632);
+            tbl[(at + 16) & 31] = __byte_perm(t2, t3, 0x5410);
+            tbl[(at + 24) & 31] = __byte_perm(t2, t3, 0x7632);
         }
         S.sum_t[slot][j][b0 + rr][bv] = tsum;
     }
@@ -415,6 +422,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
     // ======================================= MMA warps =======================================
     const int gq = lane >> 2, tq = lane & 3;
     const int w = warp;
+    const int tbl_lane = (lane & 16) | ((lane + table_rot_pairs(w)) & 15);   // this warp's tiles are j = w and w + 8: same rotation
     float sig_inv[kRed][RABIT_MAX_K];         // 1 / sigma of the batch rows this thread reduces
     {
         float sg_all[NB][RABIT_MAX_K], inv_all[NB][RABIT_MAX_K];
@@ -525,7 +533,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
 #pragma unroll
         for (int jp = 0; jp < kPairs; ++jp) {
             bb[jp] = make_uint2(0u, 0u);
-            if (2 * jp + (gq >> 2) < NB) bb[jp] = S.table[slot][j][jp * 32 + lane];
+            if (2 * jp + (gq >> 2) < NB) bb[jp] = S.table[slot][j][jp * 32 + tbl_lane];
         }
 #pragma unroll
         for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][j][b][lane & 3];   // this lane's quarter of the tile
@@ -549,7 +557,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
             const uint4 wa = S.bits[slot][w][lane];
             const uint4 wb = S.bits[slot][w + kMmaWarps][lane];
             uint2 ba = make_uint2(0u, 0u), bb = make_uint2(0u, 0u);
-            if (gq < 4 * NB) { ba = S.table[slot][w][lane]; bb = S.table[slot][w + kMmaWarps][lane]; }
+            if (gq < 4 * NB) { ba = S.table[slot][w][tbl_lane]; bb = S.table[slot][w + kMmaWarps][tbl_lane]; }
 #pragma unroll
             for (int b = 0; b < NB; ++b) sum_t[b] += S.sum_t[slot][w][b][lane & 3] + S.sum_t[slot][w + kMmaWarps][b][lane & 3];
 #pragma unroll
