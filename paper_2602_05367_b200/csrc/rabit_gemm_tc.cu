@@ -345,7 +345,7 @@ EncodeTiledFn encode_tiled_fn() {
 }  // namespace
 
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch) {
-    return batch > RABIT_MAX_GEMV_BATCH && L.geom.K <= 3 && encode_tiled_fn() != nullptr;
+    return batch >= 1 && L.geom.K <= 3 && encode_tiled_fn() != nullptr;
 }
 
 template <int TB, int KP>

@@ -59,3 +59,33 @@ def test_three_paths_large_batch():
     x = make_x(48, 256, key=(63,))
     check_against_oracle(L, x, run_layer(L, x, 0))
     check_against_oracle(L, x, run_layer(L, x, GEMM))
+
+
+@pytest.mark.parametrize("K,M,N,batch", [
+    (2, 300, 640, 1),
+    (2, 300, 640, 5),
+    (3, 200, 352, 9),
+    (2, 1000, 1184, 16),
+])
+def test_gemm_runs_small_batches_too(K, M, N, batch):
+    """The tensor-core GEMM forced onto decode-sized batches (its batch tile is then mostly zero fill)."""
+    L = make_layer(M, N, K, key=(62, K, M, N))
+    x = make_x(batch, N, key=(62, M, N, batch))
+    y = run_layer(L, x, GEMM)
+    check_against_oracle(L, x, y)
+
+
+@pytest.mark.parametrize("batch", [8, 9, 12, 16])
+def test_dispatch_between_nine_and_sixteen_rows_on_a_tall_layer(batch):
+    """A layer with many row tiles and few columns: from 9 batch rows on the dispatcher prefers one GEMM launch to
+    three or four GEMV passes.  Whichever kernel runs, the result is within tolerance and equals the forced one."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(14336, 512, 2, key=(63,))
+    x = make_x(batch, 512, key=(63, batch))
+    y_auto = run_layer(L, x, 0)
+    check_against_oracle(L, x, y_auto)
+    y_gemv = run_layer(L, x, 2)
+    y_gemm = run_layer(L, x, GEMM)
+    expect = y_gemm if batch > 8 else y_gemv
+    assert np.array_equal(y_auto.view(np.uint16), expect.view(np.uint16))
