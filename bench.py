@@ -420,6 +420,34 @@ def bench_cases(args) -> dict:
             else:
                 case["roofline"] = {"bound": "hbm", "achieved": case["gbs"], "peak": hbm_peak, "unit": "GB/s",
                                     "frac": case["gbs"] / hbm_peak}
+            if batch > 16:
+                # the same case on the dequantised-tile GEMM (variant 4: one contraction of fp16 weights instead of one per
+                # path); tflops counts the layer's algorithmic flops for both, so the two compare by time
+                for L in layers:
+                    L.set_variant(4)
+                with torch.cuda.stream(stream):
+                    for L in layers:
+                        rabit.rabit_linear(L, x, y)
+                stream.synchronize()
+                g4 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g4, stream=stream):
+                    for L in layers:
+                        rabit.rabit_linear(L, x, y)
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        g4.replay()
+                    ev0.record(stream)
+                    for _ in range(reps):
+                        g4.replay()
+                    ev1.record(stream)
+                stream.synchronize()
+                us4 = ev0.elapsed_time(ev1) * 1e3 / (reps * copies)
+                case["dequantised_tile_variant"] = {"us_per_layer": us4, "tflops_algorithmic": flops / us4 / 1e6,
+                                                    "tensor_flops_executed_tflops": flops / K_PATHS / us4 / 1e6,
+                                                    "frac_of_peak_executed": flops / K_PATHS / us4 / 1e6 / tc_peak}
+                for L in layers:
+                    L.set_variant(0)
+                del g4
             cases.append(case)
             del g
         for L in layers:

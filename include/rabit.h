@@ -216,7 +216,10 @@ RABIT_API int rabit_layer_N(const rabit_layer* layer);
 /*
  * Choose the kernel family for subsequent rabit_linear calls of this layer:
  *   0 = automatic (default), 1 = plain sign-select kernel, 2 = integer tensor-core GEMV,
- *   3 = tcgen05 GEMM.  Returns RABIT_INVALID_ARG for a variant that cannot run the layer.
+ *   3 = tcgen05 GEMM with one exact +-h_k operand tile and accumulator per path,
+ *   4 = tcgen05 GEMM on the dequantised weight tile sum_k +-g_k h_k rounded to fp16 (Eq. 2 formed per tile; one
+ *       contraction of length N instead of K of them; never chosen automatically: it rounds every weight to fp16).
+ * Returns RABIT_INVALID_ARG for a variant that cannot run the layer.
  * Meant for A/B timing and profiling; results are within tolerance for every variant.
  */
 RABIT_API int rabit_set_variant(rabit_layer* layer, int variant);

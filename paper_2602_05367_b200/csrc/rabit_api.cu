@@ -191,6 +191,11 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
                 return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: tcgen05 GEMM cannot run batch %d", batch);
             e = rabit_launch_gemm_tc(*layer, x, y, batch, st);
             break;
+        case 4:
+            if (!rabit_gemm_tc_supports(*layer, batch))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: tcgen05 GEMM cannot run batch %d", batch);
+            e = rabit_launch_gemm_tc(*layer, x, y, batch, st, true);
+            break;
         default:
             e = rabit_launch_plain(*layer, x, y, batch, st);
             break;
@@ -380,7 +385,7 @@ extern "C" int rabit_layer_N(const rabit_layer* layer) { return layer ? layer->g
 extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
-    if (variant < 0 || variant > 3) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..3");
+    if (variant < 0 || variant > 4) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..4");
     layer->variant = variant;
     return RABIT_OK;
 }

@@ -41,23 +41,23 @@ struct __align__(1024) InStage {
     __half h[KP][kStepCols];
 };
 // ... and what the expander warps make of it (two steps: one being multiplied, one being written).
-template <int KP>
+template <int KA>
 struct __align__(1024) AStage {
-    __half a[KP][kTileM * kStepCols];                 // 16 KB per path, +-h, swizzled
+    __half a[KA][kTileM * kStepCols];                 // 16 KB per expanded operand tile (one per path, or one in all), swizzled
 };
 
 // Input-ring depth: as many steps as fit beside the A ring in 222 KB, at most 8.
-template <int TB, int KP>
+template <int TB, int KP, int KA>
 struct GemmCfg {
     static constexpr int kInBytes = (int)sizeof(InStage<TB, KP>);
-    static constexpr int kFit = (222 * 1024 - kAStages * (int)sizeof(AStage<KP>)) / kInBytes;
+    static constexpr int kFit = (222 * 1024 - kAStages * (int)sizeof(AStage<KA>)) / kInBytes;
     static constexpr int kStages = kFit > 8 ? 8 : kFit;
 };
 
-template <int TB, int KP>
+template <int TB, int KP, int KA>
 struct Smem {
-    AStage<KP> astage[kAStages];
-    InStage<TB, KP> stage[GemmCfg<TB, KP>::kStages];
+    AStage<KA> astage[kAStages];
+    InStage<TB, KP> stage[GemmCfg<TB, KP, KA>::kStages];
     unsigned long long full[8];                       // TMA bytes landed (x, bits, h)
     unsigned long long empty[8];                      // MMAs that read the input stage retired
     unsigned long long a_ready[kAStages];             // expanders done
@@ -143,12 +143,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                  : "r"(taddr) : "memory");
 }
 
-template <int TB, int KP>
+// DEQ = false: one operand tile +-h_k and one accumulator per path (exact products, g_k applied in the epilogue).
+// DEQ = true:  one operand tile holding the dequantised weight sum_k +-g_k h_k rounded to fp16 and one accumulator:
+//              half the tensor-core work and half the shared-memory operand traffic, at the price of one fp16
+//              rounding per partial product and per weight (relative 2^-11 each).
+template <int TB, int KP, bool DEQ>
 __global__ void __launch_bounds__(kThreads, 1)
 rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_map) {
+    constexpr int KA = DEQ ? 1 : KP;
     using Stage = InStage<TB, KP>;
-    using Smem = Smem<TB, KP>;
-    constexpr int kStages = GemmCfg<TB, KP>::kStages;
+    using Smem = Smem<TB, KP, KA>;
+    constexpr int kStages = GemmCfg<TB, KP, KA>::kStages;
     constexpr int kTileB = TB;
     constexpr int kMaxPaths = KP;
     extern __shared__ unsigned char smem_raw[];
@@ -222,7 +227,8 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                     Stage& st = S.stage[slot];
                     const int ksub = min(2, G.n_ct - 2 * s) * 2;                                   // MMAs of K = 16 in this step (2 per column tile)
                     const uint64_t bdesc = umma_desc(smem_u32(st.x));
-                    for (int k = 0; k < K; ++k) {
+                    const int n_acc = DEQ ? 1 : K;
+                    for (int k = 0; k < n_acc; ++k) {
                         const uint64_t adesc = umma_desc(smem_u32(S.astage[aslot].a[k]));
                         for (int kk = 0; kk < ksub; ++kk)
                             umma_f16(tmem_base + (uint32_t)k * kTileB, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc,
@@ -248,13 +254,56 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         int it = 0, tile_i = 0;
         for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
+            __half2 g_rows[kMaxPaths][8];                     // DEQ: output scales of this thread's eight rows, both halves alike
+            if (DEQ) {
+#pragma unroll
+                for (int k = 0; k < kMaxPaths; ++k)
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        const int r = rt * kTileM + 16 * p + x_gq + 8 * (x_a & 1);
+                        g_rows[k][p] = __half2half2((k < K && r < G.Mp) ? P.g[(size_t)k * G.Mp + r] : __float2half(0.f));
+                    }
+            }
             for (int s = 0; s < n_steps; ++s, ++it) {
                 const int slot = it % kStages, aslot = it % kAStages;
                 mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
                 if (it >= kAStages) mbar_wait(smem_u32(&S.a_empty[aslot]), ((it / kAStages) - 1) & 1, abort_flag);
                 Stage& st = S.stage[slot];
-                AStage<KP>& ast = S.astage[aslot];
+                AStage<KA>& ast = S.astage[aslot];
                 const int cts = min(2, G.n_ct - 2 * s);
+                if (DEQ) {
+                    // dequantised operand: for each of this thread's 8 rows and 4 columns, sum_k +-g_k[row] h_k[col],
+                    // accumulated from the last (smallest) path to the first with one fused multiply-add per path
+                    uint32_t u01[kMaxPaths], u23[kMaxPaths];
+                    uint2 hv[kMaxPaths];
+#pragma unroll
+                    for (int k = 0; k < kMaxPaths; ++k) {
+                        uint32_t w = 0;
+                        hv[k] = make_uint2(0u, 0u);
+                        if (k < K && x_ct2 < cts) {
+                            w = reinterpret_cast<const uint32_t*>(&st.bits[k][x_ct2][x_l])[x_a];
+                            hv[k] = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff]);
+                        }
+                        u01[k] = __byte_perm(w, 0u, 0x1404);
+                        u23[k] = __byte_perm(w, 0u, 0x3424);
+                    }
+                    const uint32_t dst = smem_u32(ast.a[0]) + x_aoff;
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        __half2 s01 = __float2half2_rn(0.f), s23 = __float2half2_rn(0.f);
+#pragma unroll
+                        for (int k = kMaxPaths - 1; k >= 0; --k) {
+                            if (k >= K) continue;
+                            const uint32_t ox = hv[k].x ^ ((u01[k] << (7 - p)) & 0x80008000u);   // +-h: sign flipped where the weight is -1
+                            const uint32_t oy = hv[k].y ^ ((u23[k] << (7 - p)) & 0x80008000u);
+                            s01 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&ox), s01);
+                            s23 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&oy), s23);
+                        }
+                        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(*reinterpret_cast<const uint32_t*>(&s01)),
+                                     "r"(*reinterpret_cast<const uint32_t*>(&s23)) : "memory");
+                    }
+                } else
+                {
                 // This thread's packed word (column tile ct2, lane l, word a) of every path: rows 16*p + gq + 8*(a&1),
                 // columns 32*ct2 + 16*(a>>1) + 4*tq + c (c = 0..3) = bytes 0..7 of 16-byte chunk 4*ct2 + 2*(a>>1) + (tq>>1)
                 // of the row (second half if tq is odd); the chunk is XOR-swizzled with the row.
@@ -277,6 +326,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                         asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(ox), "r"(oy) : "memory");
                     }
                 }
+                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");              // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&S.a_ready[aslot]));
@@ -296,12 +346,12 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                 for (int c = 0; c < 32; ++c) v[c] = 0.f;
 #pragma unroll
                 for (int k = 0; k < kMaxPaths; ++k) {
-                    if (k >= K) break;
+                    if (k >= (DEQ ? 1 : K)) break;
                     uint32_t d[32];
                     tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(k * kTileB + col), d);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = fmaf(gk[k], __uint_as_float(d[c]), v[c]);
+                    for (int c = 0; c < 32; ++c) v[c] = DEQ ? __uint_as_float(d[c]) : fmaf(gk[k], __uint_as_float(d[c]), v[c]);
                 }
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
@@ -348,7 +398,7 @@ bool rabit_gemm_tc_supports(const rabit_layer& L, int batch) {
     return batch >= 1 && L.geom.K <= 3 && encode_tiled_fn() != nullptr;
 }
 
-template <int TB, int KP>
+template <int TB, int KP, bool DEQ>
 static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
@@ -372,21 +422,23 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
     P.n_bt = (batch + TB - 1) / TB;
     P.n_tiles = L.geom.n_rt * P.n_bt;
     static bool attr_done = false;
-    const size_t smem = sizeof(Smem<TB, KP>) + 1024;               // slack for the 1024-byte alignment of the stages
+    const size_t smem = sizeof(Smem<TB, KP, DEQ ? 1 : KP>) + 1024;               // slack for the 1024-byte alignment of the stages
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel<TB, KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel<TB, KP, DEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     int grid = L.sm_count > 0 ? L.sm_count : 148;
     if (grid > P.n_tiles) grid = P.n_tiles;
-    rabit_gemm_tc_kernel<TB, KP><<<grid, kThreads, smem, stream>>>(P, map);
+    rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
     return cudaGetLastError();
 }
 
-cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {
-    if (L.geom.K > 2) return launch_gemm<128, 3>(L, x, y, batch, stream);          // three accumulators of 128 columns
+cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised) {
+    if (dequantised)                                                                 // one accumulator: the widest batch tile for every K
+        return L.geom.K > 2 ? launch_gemm<256, 3, true>(L, x, y, batch, stream) : launch_gemm<256, 2, true>(L, x, y, batch, stream);
+    if (L.geom.K > 2) return launch_gemm<128, 3, false>(L, x, y, batch, stream);   // three accumulators of 128 columns
     // Always the widest batch tile: a tcgen05.mma of M = 128 takes about 128 clocks whatever its N (measured),
     // so narrower tiles would not shorten a step, they would only expand the signs more often.
-    return launch_gemm<256, 2>(L, x, y, batch, stream);
+    return launch_gemm<256, 2, false>(L, x, y, batch, stream);
 }

@@ -57,7 +57,7 @@ int rabit_gemv_mma_max_rows();
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream);
-cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised = false);
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch);
 
 #endif  // RABIT_INTERNAL_H_

@@ -89,3 +89,28 @@ def test_dispatch_between_nine_and_sixteen_rows_on_a_tall_layer(batch):
     y_gemm = run_layer(L, x, GEMM)
     expect = y_gemm if batch > 8 else y_gemv
     assert np.array_equal(y_auto.view(np.uint16), expect.view(np.uint16))
+
+
+DEQ = 4     # variant number of the GEMM on dequantised fp16 weight tiles
+
+
+@pytest.mark.parametrize("K,M,N,batch", [
+    (2, 128, 64, 17),
+    (1, 200, 96, 64),
+    (2, 1000, 1184, 300),
+    (2, 384, 2048, 512),
+    (3, 300, 352, 130),
+    (3, 1000, 1184, 300),
+    (2, 300, 640, 5),
+])
+def test_dequantised_tile_gemm(K, M, N, batch):
+    """Variant 4 forms sum_k +-g_k h_k per weight in fp16 and runs one contraction: every weight carries a relative
+    rounding of about 2^-11 per partial product, so the result stays inside the tolerance (worst case half of it) but is
+    not as close to the oracle as the exact-expansion GEMM."""
+    L = make_layer(M, N, K, key=(64, K, M, N))
+    x = make_x(batch, N, key=(64, M, N, batch))
+    y = run_layer(L, x, DEQ)
+    err, tol = check_against_oracle(L, x, y)
+    y_exact = run_layer(L, x, GEMM)
+    err_exact, _ = check_against_oracle(L, x, y_exact)
+    assert err_exact.max() <= err.max() + 1e-3 * tol.max()        # the exact expansion is never noticeably worse
