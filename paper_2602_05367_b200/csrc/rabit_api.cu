@@ -160,16 +160,14 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
     if (variant == 0) {
         if (batch <= RABIT_MAX_GEMV_BATCH) {
             variant = rabit_gemv_mma_supports(*layer, batch) ? 2 : 1;
-            // Between 9 and 16 batch rows the GEMV makes three or four passes over the weights; a layer with many
-            // row tiles is then cheaper on the tensor-core GEMM, whose cost does not depend on the batch up to 256.
-            // Both estimates are fits to measurements on B200 (us): a GEMV pass costs 7.6 + packed MB / 1.4, a GEMM
-            // wave (one 128-row tile per SM) 3 + 5.9 * K * N / 1024.
-            if (variant == 2 && batch > 8 && rabit_gemm_tc_supports(*layer, batch)) {
-                const int sms = layer->sm_count > 0 ? layer->sm_count : 148;
+            // From 5 batch rows on the GEMV makes two to four passes over the weights; the tensor-core GEMM, whose cost
+            // does not depend on the batch up to 256, is then often cheaper.  Both estimates are fits to measurements
+            // on B200 (us): a GEMV pass of four rows costs 10 + max(0, packed MB - 4) / 1.3.
+            if (variant == 2 && batch > 4 && rabit_gemm_tc_supports(*layer, batch)) {
                 const double passes = (double)((batch + rabit_gemv_mma_max_rows() - 1) / rabit_gemv_mma_max_rows());
-                const double gemv_us = passes * (7.6 + (double)G.K * G.Mp * G.N / 8.0 / 1.4e6);
-                const double waves = (double)((G.n_rt + sms - 1) / sms);
-                const double gemm_us = waves * (3.0 + 5.9 * G.K * (double)G.N / 1024.0);
+                const double mb = (double)G.K * G.Mp * G.N / 8.0e6;
+                const double gemv_us = passes * (10.0 + (mb > 4.0 ? (mb - 4.0) / 1.3 : 0.0));
+                const double gemm_us = rabit_gemm_tc_estimate_us(*layer, batch);
                 if (gemm_us < 0.9 * gemv_us) variant = 3;
             }
         } else {

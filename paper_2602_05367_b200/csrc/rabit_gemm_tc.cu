@@ -78,6 +78,7 @@ struct GemmParams {
     int batch;
     int n_bt;                                         // batch tiles
     int n_tiles;                                      // n_rt * n_bt
+    int split;                                        // CTAs (one cluster) that share the contraction of one tile: 1, 2, 4 or 8
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -147,6 +148,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // DEQ = true:  one operand tile holding the dequantised weight sum_k +-g_k h_k rounded to fp16 and one accumulator:
 //              half the tensor-core work and half the shared-memory operand traffic, at the price of one fp16
 //              rounding per partial product and per weight (relative 2^-11 each).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
 template <int TB, int KP, bool DEQ>
 __global__ void __launch_bounds__(kThreads, 1)
 rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_map) {
@@ -164,6 +179,16 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     const int K = G.K;
     const int n_steps = (G.N + kStepCols - 1) / kStepCols;        // N % 32 == 0: the last step may hold one column tile only
     volatile int* abort_flag = &S.abort_flag;
+    // Split contraction: the `split` CTAs of a cluster work on the same output tile, rank r taking the r-th part of
+    // the 64-column steps; their partial results meet through distributed shared memory at the end.  Each CTA
+    // then has exactly one tile.  split == 1 is the persistent form (a CTA walks tiles blockIdx.x, +gridDim.x, ...).
+    const int split = P.split;
+    uint32_t crank = 0;
+    if (split > 1) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+    const int t_first = split > 1 ? (int)blockIdx.x / split : (int)blockIdx.x;
+    const int t_stride = split > 1 ? P.n_tiles : (int)gridDim.x;
+    const int s_lo = split > 1 ? (int)((long long)n_steps * crank / split) : 0;
+    const int s_hi = split > 1 ? (int)((long long)n_steps * (crank + 1) / split) : n_steps;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -192,9 +217,9 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         // ===================================== producer =====================================
         if (lane == 0) {
             int it = 0;                                          // global step counter of this CTA
-            for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x) {
+            for (int t = t_first; t < P.n_tiles; t += t_stride) {
                 const int rt = t / P.n_bt, bt = t % P.n_bt;
-                for (int s = 0; s < n_steps; ++s, ++it) {
+                for (int s = s_lo; s < s_hi; ++s, ++it) {
                     const int slot = it % kStages;
                     if (it >= kStages) mbar_wait(smem_u32(&S.empty[slot]), ((it / kStages) - 1) & 1, abort_flag);
                     Stage& st = S.stage[slot];
@@ -216,10 +241,10 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(kTileB);
             int it = 0, tile_i = 0;
-            for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
+            for (int t = t_first; t < P.n_tiles; t += t_stride, ++tile_i) {
                 if (tile_i > 0) mbar_wait(smem_u32(&S.acc_empty), (tile_i - 1) & 1, abort_flag);   // epilogue has drained the accumulators
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                for (int s = 0; s < n_steps; ++s, ++it) {
+                for (int s = s_lo; s < s_hi; ++s, ++it) {
                     const int slot = it % kStages, aslot = it % kAStages;
                     mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
                     mbar_wait(smem_u32(&S.a_ready[aslot]), (it / kAStages) & 1, abort_flag);
@@ -232,7 +257,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                         const uint64_t adesc = umma_desc(smem_u32(S.astage[aslot].a[k]));
                         for (int kk = 0; kk < ksub; ++kk)
                             umma_f16(tmem_base + (uint32_t)k * kTileB, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc,
-                                     (s > 0 || kk > 0) ? 1u : 0u);
+                                     (s > s_lo || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&S.empty[slot]));                                         // frees both stages when these MMAs retire
                     umma_commit(smem_u32(&S.a_empty[aslot]));
@@ -252,7 +277,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
         const uint32_t x_aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
         int it = 0, tile_i = 0;
-        for (int t = blockIdx.x; t < P.n_tiles; t += gridDim.x, ++tile_i) {
+        for (int t = t_first; t < P.n_tiles; t += t_stride, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
             __half2 g_rows[kMaxPaths][8];                     // DEQ: output scales of this thread's eight rows, both halves alike
             if (DEQ) {
@@ -264,7 +289,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                         g_rows[k][p] = __half2half2((k < K && r < G.Mp) ? P.g[(size_t)k * G.Mp + r] : __float2half(0.f));
                     }
             }
-            for (int s = 0; s < n_steps; ++s, ++it) {
+            for (int s = s_lo; s < s_hi; ++s, ++it) {
                 const int slot = it % kStages, aslot = it % kAStages;
                 mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
                 if (it >= kAStages) mbar_wait(smem_u32(&S.a_empty[aslot]), ((it / kAStages) - 1) & 1, abort_flag);
@@ -331,6 +356,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&S.a_ready[aslot]));
             }
+            if (split > 1) break;                              // the cluster's epilogue follows the role branches
             // ---- epilogue of this tile
             mbar_wait(smem_u32(&S.acc_ready), tile_i & 1, abort_flag);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -365,6 +391,66 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         }
     }
 
+    if (split > 1) {
+        // ---- epilogue of a split tile.  Every CTA of the cluster holds a partial 128 x TB result in tensor memory.
+        //      CTA `o` finishes the batch columns [o*W, (o+1)*W), W = TB / split: all CTAs send it their slice of
+        //      those columns (already scaled by g_k and summed over the paths), into its receive buffer
+        //      recv[source rank][column][row] (the input ring's memory: nothing uses it once every CTA's MMAs have
+        //      retired, which the first cluster barrier establishes).  After the second barrier each CTA adds the
+        //      slices it received in rank order and stores fp16.
+        const int rt = t_first / P.n_bt, bt = t_first % P.n_bt;
+        const int W = kTileB / split;
+        if (warp >= 2) {
+            mbar_wait(smem_u32(&S.acc_ready), 0, abort_flag);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        __syncwarp();
+        cluster_sync_all();
+        float* recv = reinterpret_cast<float*>(&S.stage[0]);
+        if (warp >= 2) {
+            const int e = warp - 2, quarter = warp & 3, col_half = e >> 2;
+            const int r_in = quarter * 32 + lane;                                  // row of the tile this thread reads from tensor memory
+            const int row = rt * kTileM + r_in;
+            float gk[kMaxPaths];
+#pragma unroll
+            for (int k = 0; k < kMaxPaths; ++k) gk[k] = (k < K && row < G.Mp) ? __half2float(P.g[(size_t)k * G.Mp + row]) : 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kTileB / 2; c0 += 32) {
+                const int col = col_half * (kTileB / 2) + c0;
+                float v[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] = 0.f;
+#pragma unroll
+                for (int k = 0; k < kMaxPaths; ++k) {
+                    if (k >= (DEQ ? 1 : K)) break;
+                    uint32_t d[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(k * kTileB + col), d);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) v[c] = DEQ ? __uint_as_float(d[c]) : fmaf(gk[k], __uint_as_float(d[c]), v[c]);
+                }
+                const int owner = col / W, lc0 = col % W;                         // 32 divides W: the chunk has one owner
+                const uint32_t dst = cluster_map(smem_u32(recv + ((size_t)crank * W + lc0) * kTileM + r_in), (uint32_t)owner);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) st_cluster_f32(dst + (uint32_t)(c * kTileM * 4), v[c]);
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        }
+        __syncwarp();
+        cluster_sync_all();
+        if (warp >= 2) {
+            const int et = (warp - 2) * 32 + lane;
+            const int r_in = et & (kTileM - 1), hh = et >> 7;                     // two threads per row, half of the W columns each
+            const int row = rt * kTileM + r_in;
+            for (int lc = hh * (W / 2); lc < (hh + 1) * (W / 2); ++lc) {
+                float sum = 0.f;
+                for (int src = 0; src < split; ++src) sum += recv[((size_t)src * W + lc) * kTileM + r_in];
+                const int b = bt * kTileB + (int)crank * W + lc;
+                if (b < P.batch && row < G.M) P.y[(size_t)b * G.M + row] = __float2half_rn(sum);
+            }
+        }
+    }
+
     // ---- teardown: everyone meets, then the allocating warp frees the tensor memory
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -393,6 +479,27 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 }  // namespace
+
+// CTAs per cluster that share one tile's contraction: doubled while every CTA keeps at least 8 steps, the
+// slices stay 32 columns wide and the whole grid is resident at once.
+static int choose_split(int n_tiles, int N, int tb, int sms) {
+    const int n_steps = (N + kStepCols - 1) / kStepCols;
+    int split = 1;
+    while (split < 8 && n_tiles * split * 2 <= sms && n_steps / (split * 2) >= 8 && tb / (split * 2) >= 32) split *= 2;
+    return split;
+}
+
+// Estimated duration (us) of the exact-expansion GEMM on B200, a fit to measurements at batch <= 64:
+// 11 + 0.75 * (K/2) per 64-column step of the busiest CTA, times the number of waves.
+double rabit_gemm_tc_estimate_us(const rabit_layer& L, int batch) {
+    const int sms = L.sm_count > 0 ? L.sm_count : 148;
+    const int tb = L.geom.K > 2 ? 128 : 256;
+    const int n_tiles = L.geom.n_rt * ((batch + tb - 1) / tb);
+    const int split = choose_split(n_tiles, L.geom.N, tb, sms);
+    const int n_steps = (L.geom.N + kStepCols - 1) / kStepCols;
+    const double waves = split > 1 ? 1.0 : (double)((n_tiles + sms - 1) / sms);
+    return waves * (11.0 + 0.375 * L.geom.K * (double)((n_steps + split - 1) / split));
+}
 
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch) {
     return batch >= 1 && L.geom.K <= 3 && encode_tiled_fn() != nullptr;
@@ -428,10 +535,31 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    int grid = L.sm_count > 0 ? L.sm_count : 148;
+    const int sms = L.sm_count > 0 ? L.sm_count : 148;
+    int grid = sms;
     if (grid > P.n_tiles) grid = P.n_tiles;
-    rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
-    return cudaGetLastError();
+    // Few tiles (a layer with few rows, or a batch of one tile): the CTAs of a cluster share each tile's contraction
+    // as long as every CTA keeps at least 8 steps, the slices stay 32 columns wide and the whole grid is resident.
+    int split = choose_split(P.n_tiles, L.geom.N, TB, sms);
+    if (sizeof(InStage<TB, KP>) * GemmCfg<TB, KP, DEQ ? 1 : KP>::kStages < (size_t)kTileM * TB * 4) split = 1;   // the receive buffer lives in the input ring
+    P.split = split;
+    if (split == 1) {
+        rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned int)(P.n_tiles * split));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned int)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rabit_gemm_tc_kernel<TB, KP, DEQ>, P, map);
 }
 
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised) {

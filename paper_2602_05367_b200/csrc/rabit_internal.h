@@ -59,5 +59,6 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
                                         int batch, cudaStream_t stream);
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised = false);
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch);
+double rabit_gemm_tc_estimate_us(const rabit_layer& L, int batch);
 
 #endif  // RABIT_INTERNAL_H_

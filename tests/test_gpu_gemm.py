@@ -75,20 +75,24 @@ def test_gemm_runs_small_batches_too(K, M, N, batch):
     check_against_oracle(L, x, y)
 
 
-@pytest.mark.parametrize("batch", [8, 9, 12, 16])
-def test_dispatch_between_nine_and_sixteen_rows_on_a_tall_layer(batch):
-    """A layer with many row tiles and few columns: from 9 batch rows on the dispatcher prefers one GEMM launch to
-    three or four GEMV passes.  Whichever kernel runs, the result is within tolerance and equals the forced one."""
-    import torch
-    import paper_2602_05367_b200 as rabit
+@pytest.mark.parametrize("batch", [4, 8, 12, 16])
+def test_dispatch_between_five_and_sixteen_rows(batch):
+    """Up to four batch rows always take the GEMV (one pass); beyond that the dispatcher compares its cost estimates of
+    the GEMV passes and of one GEMM launch.  Whichever kernel runs, the result is within tolerance and is exactly what
+    that kernel gives when forced; on this tall, narrow layer 16 rows go to the GEMM."""
     L = make_layer(14336, 512, 2, key=(63,))
     x = make_x(batch, 512, key=(63, batch))
     y_auto = run_layer(L, x, 0)
     check_against_oracle(L, x, y_auto)
     y_gemv = run_layer(L, x, 2)
     y_gemm = run_layer(L, x, GEMM)
-    expect = y_gemm if batch > 8 else y_gemv
-    assert np.array_equal(y_auto.view(np.uint16), expect.view(np.uint16))
+    same_gemv = np.array_equal(y_auto.view(np.uint16), y_gemv.view(np.uint16))
+    same_gemm = np.array_equal(y_auto.view(np.uint16), y_gemm.view(np.uint16))
+    assert same_gemv or same_gemm
+    if batch <= 4:
+        assert same_gemv
+    if batch == 16:
+        assert same_gemm
 
 
 DEQ = 4     # variant number of the GEMM on dequantised fp16 weight tiles
@@ -114,3 +118,29 @@ def test_dequantised_tile_gemm(K, M, N, batch):
     y_exact = run_layer(L, x, GEMM)
     err_exact, _ = check_against_oracle(L, x, y_exact)
     assert err_exact.max() <= err.max() + 1e-3 * tol.max()        # the exact expansion is never noticeably worse
+
+
+@pytest.mark.parametrize("K,M,N,batch,variant", [
+    (2, 256, 4096, 64, GEMM),      # 2 tiles, 64 steps: eight CTAs share a tile (32-column slices)
+    (2, 256, 4096, 300, GEMM),     # two batch tiles, ragged
+    (2, 200, 4160, 40, DEQ),       # ragged rows, 65 steps split unevenly
+    (3, 256, 2048, 100, GEMM),     # three paths: 128-wide tiles, four CTAs per tile
+    (1, 384, 1024, 17, GEMM),      # two CTAs per tile
+    (2, 1024, 8192, 512, GEMM),    # the 70B k/v projection at batch 512: 16 tiles, eight CTAs each
+])
+def test_gemm_split_contraction_across_a_cluster(K, M, N, batch, variant):
+    """Layers with few output tiles: the CTAs of a cluster split the contraction of a tile and add their partial
+    results through distributed shared memory (fixed order, so the result is deterministic)."""
+    L = make_layer(M, N, K, key=(65, K, M, N))
+    x = make_x(batch, N, key=(65, M, N, batch))
+    y = run_layer(L, x, variant)
+    if M * N * batch <= 2 ** 31:
+        check_against_oracle(L, x, y)
+    else:                                           # large case: sampled rows
+        rows = np.unique(np.concatenate([np.arange(0, 4), np.arange(126, 131), np.arange(M - 3, M), np.random.default_rng(0).integers(0, M, 24)]))
+        from oracle import rabit_oracle as orc
+        ref = orc.linear(L.planes[:, rows, :], L.g[:, rows], L.h, x)
+        tol = orc.tolerance(L.g, L.h, x)
+        assert (np.abs(y[:, rows].astype(np.float64) - ref).max(axis=1) <= tol).all()
+    y2 = run_layer(L, x, variant)
+    assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
