@@ -559,7 +559,11 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rabit_gemm_tc_kernel<TB, KP, DEQ>, P, map);
+    if (cudaLaunchKernelEx(&cfg, rabit_gemm_tc_kernel<TB, KP, DEQ>, P, map) == cudaSuccess) return cudaSuccess;
+    cudaGetLastError();                                            // clusters of this size cannot be placed here: one CTA per tile instead
+    P.split = 1;
+    rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
+    return cudaGetLastError();
 }
 
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised) {
