@@ -77,7 +77,7 @@ struct GemmParams {
     unsigned int* status;
     int batch;
     int n_bt;                                         // batch tiles
-    int n_tiles;                                      // n_rt * n_bt
+    int tile_lo, tile_hi;                             // this launch covers tiles tile_lo .. tile_hi - 1 of the n_rt * n_bt
     int split;                                        // CTAs (one cluster) that share the contraction of one tile: 1, 2, 4 or 8
 };
 
@@ -185,8 +185,8 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     const int split = P.split;
     uint32_t crank = 0;
     if (split > 1) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
-    const int t_first = split > 1 ? (int)blockIdx.x / split : (int)blockIdx.x;
-    const int t_stride = split > 1 ? P.n_tiles : (int)gridDim.x;
+    const int t_first = P.tile_lo + (split > 1 ? (int)blockIdx.x / split : (int)blockIdx.x);
+    const int t_stride = split > 1 ? P.tile_hi - P.tile_lo : (int)gridDim.x;
     const int s_lo = split > 1 ? (int)((long long)n_steps * crank / split) : 0;
     const int s_hi = split > 1 ? (int)((long long)n_steps * (crank + 1) / split) : n_steps;
 
@@ -217,7 +217,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         // ===================================== producer =====================================
         if (lane == 0) {
             int it = 0;                                          // global step counter of this CTA
-            for (int t = t_first; t < P.n_tiles; t += t_stride) {
+            for (int t = t_first; t < P.tile_hi; t += t_stride) {
                 const int rt = t / P.n_bt, bt = t % P.n_bt;
                 for (int s = s_lo; s < s_hi; ++s, ++it) {
                     const int slot = it % kStages;
@@ -241,7 +241,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(kTileB);
             int it = 0, tile_i = 0;
-            for (int t = t_first; t < P.n_tiles; t += t_stride, ++tile_i) {
+            for (int t = t_first; t < P.tile_hi; t += t_stride, ++tile_i) {
                 if (tile_i > 0) mbar_wait(smem_u32(&S.acc_empty), (tile_i - 1) & 1, abort_flag);   // epilogue has drained the accumulators
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int s = s_lo; s < s_hi; ++s, ++it) {
@@ -277,7 +277,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
         const uint32_t x_aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
         int it = 0, tile_i = 0;
-        for (int t = t_first; t < P.n_tiles; t += t_stride, ++tile_i) {
+        for (int t = t_first; t < P.tile_hi; t += t_stride, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
             __half2 g_rows[kMaxPaths][8];                     // DEQ: output scales of this thread's eight rows, both halves alike
             if (DEQ) {
@@ -527,7 +527,7 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
     P.status = L.d_status;
     P.batch = batch;
     P.n_bt = (batch + TB - 1) / TB;
-    P.n_tiles = L.geom.n_rt * P.n_bt;
+    const int n_tiles = L.geom.n_rt * P.n_bt;
     static bool attr_done = false;
     const size_t smem = sizeof(Smem<TB, KP, DEQ ? 1 : KP>) + 1024;               // slack for the 1024-byte alignment of the stages
     if (!attr_done) {
@@ -536,34 +536,45 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
         attr_done = true;
     }
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
-    int grid = sms;
-    if (grid > P.n_tiles) grid = P.n_tiles;
-    // Few tiles (a layer with few rows, or a batch of one tile): the CTAs of a cluster share each tile's contraction
-    // as long as every CTA keeps at least 8 steps, the slices stay 32 columns wide and the whole grid is resident.
-    int split = choose_split(P.n_tiles, L.geom.N, TB, sms);
-    if (sizeof(InStage<TB, KP>) * GemmCfg<TB, KP, DEQ ? 1 : KP>::kStages < (size_t)kTileM * TB * 4) split = 1;   // the receive buffer lives in the input ring
-    P.split = split;
-    if (split == 1) {
-        rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
+    const bool ring_holds_exchange = sizeof(InStage<TB, KP>) * GemmCfg<TB, KP, DEQ ? 1 : KP>::kStages >= (size_t)kTileM * TB * 4;   // the receive buffer lives in the input ring
+
+    // One launch over tiles [lo, hi).  Few tiles: the CTAs of a cluster share each tile's contraction (see choose_split).
+    auto launch_range = [&](int lo, int hi) -> cudaError_t {
+        GemmParams Q = P;
+        Q.tile_lo = lo;
+        Q.tile_hi = hi;
+        const int count = hi - lo;
+        int grid = sms < count ? sms : count;
+        int split = ring_holds_exchange ? choose_split(count, L.geom.N, TB, sms) : 1;
+        Q.split = split;
+        if (split > 1) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned int)(count * split));
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned int)split;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, rabit_gemm_tc_kernel<TB, KP, DEQ>, Q, map) == cudaSuccess) return cudaSuccess;
+            cudaGetLastError();                                    // clusters of this size cannot be placed here: one CTA per tile instead
+            Q.split = 1;
+        }
+        rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(Q, map);
         return cudaGetLastError();
+    };
+    // A few tiles beyond whole waves would cost a whole wave of their own: they go to a second, split launch.
+    const int whole = (n_tiles / sms) * sms, rest = n_tiles - whole;
+    if (whole > 0 && rest > 0 && ring_holds_exchange && choose_split(rest, L.geom.N, TB, sms) >= 2) {
+        cudaError_t e = launch_range(0, whole);
+        if (e != cudaSuccess) return e;
+        return launch_range(whole, n_tiles);
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned int)(P.n_tiles * split));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned int)split;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, rabit_gemm_tc_kernel<TB, KP, DEQ>, P, map) == cudaSuccess) return cudaSuccess;
-    cudaGetLastError();                                            // clusters of this size cannot be placed here: one CTA per tile instead
-    P.split = 1;
-    rabit_gemm_tc_kernel<TB, KP, DEQ><<<grid, kThreads, smem, stream>>>(P, map);
-    return cudaGetLastError();
+    return launch_range(0, n_tiles);
 }
 
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised) {
