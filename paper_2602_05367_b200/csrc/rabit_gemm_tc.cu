@@ -482,11 +482,18 @@ EncodeTiledFn encode_tiled_fn() {
 
 // CTAs per cluster that share one tile's contraction: doubled while every CTA keeps at least 8 steps, the
 // slices stay 32 columns wide and the whole grid is resident at once.
+// Clusters of 2 / 4 / 8 of these one-per-SM CTAs that the device places at once (index log2 of the size); cautious
+// defaults until a launch has asked the runtime (a cluster must sit inside one GPC, so 8-CTA clusters are few).
+static int g_cluster_limit[4] = {1 << 30, 64, 28, 8};
+
 static int choose_split(int n_tiles, int N, int tb, int sms) {
     const int n_steps = (N + kStepCols - 1) / kStepCols;
-    int split = 1;
-    while (split < 8 && n_tiles * split * 2 <= sms && n_steps / (split * 2) >= 8 && tb / (split * 2) >= 32) split *= 2;
-    return split;
+    int best = 1;
+    for (int lg = 1; lg <= 3; ++lg) {
+        const int split = 1 << lg;
+        if (n_tiles * split <= sms && n_tiles <= g_cluster_limit[lg] && n_steps / split >= 8 && tb / split >= 32) best = split;
+    }
+    return best;
 }
 
 // Estimated duration (us) of the exact-expansion GEMM on B200, a fit to measurements at batch <= 64:
@@ -537,6 +544,27 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
     }
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
     const bool ring_holds_exchange = sizeof(InStage<TB, KP>) * GemmCfg<TB, KP, DEQ ? 1 : KP>::kStages >= (size_t)kTileM * TB * 4;   // the receive buffer lives in the input ring
+
+    static bool limits_done = false;
+    if (!limits_done) {                                            // how many clusters of each size fit at once (asked once per kernel)
+        for (int lg = 1; lg <= 3; ++lg) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3((unsigned int)((sms / (1 << lg)) * (1 << lg)));
+            q.blockDim = dim3(kThreads);
+            q.dynamicSmemBytes = smem;
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 1u << lg;
+            qa[0].val.clusterDim.y = 1;
+            qa[0].val.clusterDim.z = 1;
+            q.attrs = qa;
+            q.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, rabit_gemm_tc_kernel<TB, KP, DEQ>, &q) == cudaSuccess && n > 0) g_cluster_limit[lg] = n;
+            else cudaGetLastError();
+        }
+        limits_done = true;
+    }
 
     // One launch over tiles [lo, hi).  Few tiles: the CTAs of a cluster share each tile's contraction (see choose_split).
     auto launch_range = [&](int lo, int hi) -> cudaError_t {
