@@ -1,4 +1,4 @@
-// Large-batch form of the layer on the tcgen05 tensor cores (batch > 16).
+// Large-batch form of the layer on the tcgen05 tensor cores (batch > 16, and smaller batches where it is cheaper).
 //
 //   y[b][i] = sum_k g_k[i] * sum_j (B_k[i][j] * h_k[j]) * x[b][j]                       (Section 4.1, Eq. 2)
 //
@@ -17,6 +17,13 @@
 //               (same warps) read the accumulators with tcgen05.ld for the epilogue
 // Every wait is bounded; on a time-out the CTA sets the status word, skips the remaining waits,
 // frees its tensor memory and returns.
+//
+// Two more forms of the same kernel:
+//   * split contraction: when a launch has fewer tiles than half the SMs, clusters of 2, 4 or 8 CTAs share the 64-column
+//     steps of one tile and add their partial results through distributed shared memory (fixed order, no atomics);
+//     tiles left over beyond whole waves of the persistent form are launched that way too;
+//   * DEQ: the expander forms the dequantised weight sum_k +-g_k h_k in fp16 and one contraction serves all paths
+//     (rabit_set_variant 4; half the tensor work, one fp16 rounding per partial product and weight).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
