@@ -35,7 +35,9 @@ constexpr int kTileM = 128;                 // weight rows per output tile
 // batch rows per output tile (MMA N) and paths: TB = 256 with up to 2 paths or TB = 128 with 3 (template parameters):
 // paths x TB accumulator columns must fit the 512 columns of tensor memory
 constexpr int kStepCols = 64;               // input columns per pipeline step (128 bytes of fp16: one swizzle row)
-constexpr int kAStages = 2;                 // expanded A tiles are double-buffered
+// Expanded A tiles: double-buffered, or four stages where there is one tile per step (KA == 1, the dequantised form),
+// whose expander warps work as two groups on alternate steps.
+__host__ __device__ constexpr int a_stages(int ka) { return ka == 1 ? 4 : 2; }
 constexpr int kExpandWarps = 8;
 constexpr int kThreads = (2 + kExpandWarps) * 32;
 constexpr long long kWaitLimitCycles = 1LL << 31;
@@ -57,18 +59,18 @@ struct __align__(1024) AStage {
 template <int TB, int KP, int KA>
 struct GemmCfg {
     static constexpr int kInBytes = (int)sizeof(InStage<TB, KP>);
-    static constexpr int kFit = (222 * 1024 - kAStages * (int)sizeof(AStage<KA>)) / kInBytes;
+    static constexpr int kFit = (222 * 1024 - a_stages(KA) * (int)sizeof(AStage<KA>)) / kInBytes;
     static constexpr int kStages = kFit > 8 ? 8 : kFit;
 };
 
 template <int TB, int KP, int KA>
 struct Smem {
-    AStage<KA> astage[kAStages];
+    AStage<KA> astage[a_stages(KA)];
     InStage<TB, KP> stage[GemmCfg<TB, KP, KA>::kStages];
     unsigned long long full[8];                       // TMA bytes landed (x, bits, h)
     unsigned long long empty[8];                      // MMAs that read the input stage retired
-    unsigned long long a_ready[kAStages];             // expanders done
-    unsigned long long a_empty[kAStages];             // MMAs that read the A stage retired
+    unsigned long long a_ready[4];                    // expanders done (a_stages(KA) in use)
+    unsigned long long a_empty[4];                    // MMAs that read the A stage retired
     unsigned long long acc_ready;                     // all MMAs of the tile retired
     unsigned long long acc_empty;                     // epilogue has read the accumulators
     uint32_t tmem_base;
@@ -176,6 +178,8 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     using Stage = InStage<TB, KP>;
     using Smem = Smem<TB, KP, KA>;
     constexpr int kStages = GemmCfg<TB, KP, KA>::kStages;
+    constexpr int kAStages = a_stages(KA);
+    constexpr int kGroupWarps = DEQ ? kExpandWarps / 2 : kExpandWarps;   // expander warps that build one step's operand
     constexpr int kTileB = TB;
     constexpr int kMaxPaths = KP;
     extern __shared__ unsigned char smem_raw[];
@@ -203,7 +207,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
             mbar_init(smem_u32(&S.empty[s]), 1);
         }
         for (int s = 0; s < kAStages; ++s) {
-            mbar_init(smem_u32(&S.a_ready[s]), kExpandWarps);
+            mbar_init(smem_u32(&S.a_ready[s]), kGroupWarps);
             mbar_init(smem_u32(&S.a_empty[s]), 1);
         }
         mbar_init(smem_u32(&S.acc_ready), 1);
@@ -279,7 +283,10 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int quarter = warp & 3;                         // tensor-memory lanes this warp may read: 32*quarter .. +31
         const int col_half = e >> 2;                          // which half of the tile's batch columns this warp drains
         // expander role of this thread, the same in every step: one packed word position per path
-        const int x_ct2 = et >> 7, x_l = (et >> 2) & 31, x_a = et & 3;
+        // (dequantised form: the warps are two groups that take alternate steps; a thread then covers both column tiles of its step)
+        const int grp = e >> 2;
+        const int pos = DEQ ? ((e & 3) * 32 + lane) : et;
+        const int x_ct2 = DEQ ? 0 : et >> 7, x_l = (pos >> 2) & 31, x_a = pos & 3;
         const int x_gq = x_l >> 2, x_tq = x_l & 3;
         const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
         const uint32_t x_aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
@@ -297,6 +304,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                     }
             }
             for (int s = s_lo; s < s_hi; ++s, ++it) {
+                if (DEQ && (it & 1) != grp) continue;                 // the other group's step
                 const int slot = it % kStages, aslot = it % kAStages;
                 mbar_wait(smem_u32(&S.full[slot]), (it / kStages) & 1, abort_flag);
                 if (it >= kAStages) mbar_wait(smem_u32(&S.a_empty[aslot]), ((it / kAStages) - 1) & 1, abort_flag);
@@ -306,33 +314,39 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                 if (DEQ) {
                     // dequantised operand: for each of this thread's 8 rows and 4 columns, sum_k +-g_k[row] h_k[col],
                     // accumulated from the last (smallest) path to the first with one fused multiply-add per path
-                    uint32_t u01[kMaxPaths], u23[kMaxPaths];
-                    uint2 hv[kMaxPaths];
 #pragma unroll
-                    for (int k = 0; k < kMaxPaths; ++k) {
-                        uint32_t w = 0;
-                        hv[k] = make_uint2(0u, 0u);
-                        if (k < K && x_ct2 < cts) {
-                            w = reinterpret_cast<const uint32_t*>(&st.bits[k][x_ct2][x_l])[x_a];
-                            hv[k] = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff]);
+                    for (int ct2 = 0; ct2 < 2; ++ct2) {
+                        if (ct2 >= cts) break;
+                        uint32_t u01[kMaxPaths], u23[kMaxPaths];
+                        uint2 hv[kMaxPaths];
+#pragma unroll
+                        for (int k = 0; k < kMaxPaths; ++k) {
+                            uint32_t w = 0;
+                            hv[k] = make_uint2(0u, 0u);
+                            if (k < K) {
+                                w = reinterpret_cast<const uint32_t*>(&st.bits[k][ct2][x_l])[x_a];
+                                hv[k] = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff + 32 * ct2]);
+                            }
+                            u01[k] = __byte_perm(w, 0u, 0x1404);
+                            u23[k] = __byte_perm(w, 0u, 0x3424);
                         }
-                        u01[k] = __byte_perm(w, 0u, 0x1404);
-                        u23[k] = __byte_perm(w, 0u, 0x3424);
-                    }
-                    const uint32_t dst = smem_u32(ast.a[0]) + x_aoff;
+                        // the 16-byte chunk index of the row gains 4 per column tile before the XOR swizzle
+                        const uint32_t aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
+                        const uint32_t dst = smem_u32(ast.a[0]) + aoff;
 #pragma unroll
-                    for (int p = 0; p < 8; ++p) {
-                        __half2 s01 = __float2half2_rn(0.f), s23 = __float2half2_rn(0.f);
+                        for (int p = 0; p < 8; ++p) {
+                            __half2 s01 = __float2half2_rn(0.f), s23 = __float2half2_rn(0.f);
 #pragma unroll
-                        for (int k = kMaxPaths - 1; k >= 0; --k) {
-                            if (k >= K) continue;
-                            const uint32_t ox = hv[k].x ^ ((u01[k] << (7 - p)) & 0x80008000u);   // +-h: sign flipped where the weight is -1
-                            const uint32_t oy = hv[k].y ^ ((u23[k] << (7 - p)) & 0x80008000u);
-                            s01 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&ox), s01);
-                            s23 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&oy), s23);
+                            for (int k = kMaxPaths - 1; k >= 0; --k) {
+                                if (k >= K) continue;
+                                const uint32_t ox = hv[k].x ^ ((u01[k] << (7 - p)) & 0x80008000u);   // +-h: sign flipped where the weight is -1
+                                const uint32_t oy = hv[k].y ^ ((u23[k] << (7 - p)) & 0x80008000u);
+                                s01 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&ox), s01);
+                                s23 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&oy), s23);
+                            }
+                            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(*reinterpret_cast<const uint32_t*>(&s01)),
+                                         "r"(*reinterpret_cast<const uint32_t*>(&s23)) : "memory");
                         }
-                        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(*reinterpret_cast<const uint32_t*>(&s01)),
-                                     "r"(*reinterpret_cast<const uint32_t*>(&s23)) : "memory");
                     }
                 } else
                 {
