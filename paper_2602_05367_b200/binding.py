@@ -151,6 +151,8 @@ class RabitLayer:
         return self._handle
 
     def set_variant(self, variant: int) -> None:
+        """Kernel family for later rabit_linear calls of this layer: 0 automatic, 1 plain, 2 integer tensor-core GEMV,
+        3 tcgen05 GEMM (exact expansion), 4 tcgen05 GEMM on dequantised fp16 weight tiles (never chosen automatically)."""
         _check(_lib.rabit_set_variant(self.handle, variant))
 
     def status(self, clear: bool = False, stream: int = 0) -> int:
