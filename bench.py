@@ -357,6 +357,7 @@ def bench_cases(args) -> dict:
     """Extra workloads (not the default line): one (shape, batch) case at a time, rotating over enough
     distinct copies of the layer to exceed L2, CUDA-graph replay, CUDA-event timing.
       gemm70b : 70B-shaped layers at batch 512 (tensor-core GEMM), roofline = measured bf16 TFLOP/s
+      gemm7b  : the three distinct 7B-shaped layers at batch 128, 512 and 2048 (prefill sizes; split and whole-wave launches)
       gemv70b : the same layers at batch 1 (HBM roofline)
       sweep8b : Llama-3-8B shapes at batch 1,2,4,8,16 (HBM roofline per batch)"""
     import torch
@@ -371,6 +372,13 @@ def bench_cases(args) -> dict:
             if (sh.M, sh.N) not in seen:
                 seen.add((sh.M, sh.N)); shapes.append(sh)
         batches, cfg = [1, 2, 4, 8, 16], 3
+    elif args.workload == "gemm7b":
+        from synth import llama2_7b_layer_shapes
+        seen, shapes = set(), []
+        for sh in llama2_7b_layer_shapes():
+            if (sh.M, sh.N) not in seen:
+                seen.add((sh.M, sh.N)); shapes.append(sh)
+        batches, cfg = [128, 512, 2048], 1
     else:
         shapes, cfg = llama_70b_layer_shapes(), 4
         batches = [512] if args.workload == "gemm70b" else [1]
@@ -457,8 +465,8 @@ def bench_cases(args) -> dict:
     clocks = sampler.summary(t_start, time.time())
     sampler.stop()
     head = max(cases, key=lambda c: c["M"] * c["N"] * c["batch"])
-    gemm = args.workload == "gemm70b"
-    return {"metric": "batch-512 residual-binary GEMM TFLOP/s" if gemm else METRIC,
+    gemm = args.workload in ("gemm70b", "gemm7b")
+    return {"metric": ("batch-512 residual-binary GEMM TFLOP/s" if args.workload == "gemm70b" else "residual-binary GEMM TFLOP/s (largest case)") if gemm else METRIC,
             "value": head["tflops"] if gemm else head["us_per_layer"], "unit": "TFLOP/s" if gemm else UNIT,
             "n_gpus": 1, "steps": args.steps, "warmup": 3, "ms_per_step": head["us_per_layer"] / 1e3,
             "higher_is_better": gemm, "scaling": "weak", "vs_baseline": None,
@@ -561,7 +569,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-group", action="store_true", help="one rabit_linear launch per projection (7 per step instead of 4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemv70b", "sweep8b", "derive7b"],
+    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemm7b", "gemv70b", "sweep8b", "derive7b"],
                     help="decoder7b is the contract's line; the others are extra single-GPU measurements")
     args = ap.parse_args()
     if args.warmup < 3:
