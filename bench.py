@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) of the four launches of one grouped step, from the ncu capture summarised in
 # profiles/gemv_mma_llama2_7b_decoder_layer.md (12.759 + 4.296 + 22.771 + 11.417 MB); valid for the
 # default grouped batch-1 workload only.
-NCU_DRAM_BYTES_PER_GROUPED_STEP = 51_275_264
+NCU_DRAM_BYTES_PER_GROUPED_STEP = 51_272_192
 
 METRIC = "batch-1 residual-binary GEMV us/layer"
 UNIT = "us/layer"
