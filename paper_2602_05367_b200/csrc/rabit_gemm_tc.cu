@@ -279,29 +279,36 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
     } else {
         // ============================ expanders, then epilogue ============================
         const int e = warp - 2;                               // 0..7
-        const int et = e * 32 + lane;                         // 0..255
         const int quarter = warp & 3;                         // tensor-memory lanes this warp may read: 32*quarter .. +31
         const int col_half = e >> 2;                          // which half of the tile's batch columns this warp drains
         // expander role of this thread, the same in every step: one packed word position per path
         // (dequantised form: the warps are two groups that take alternate steps; a thread then covers both column tiles of its step)
         const int grp = e >> 2;
-        const int pos = DEQ ? ((e & 3) * 32 + lane) : et;
-        const int x_ct2 = DEQ ? 0 : et >> 7, x_l = (pos >> 2) & 31, x_a = pos & 3;
-        const int x_gq = x_l >> 2, x_tq = x_l & 3;
+        // Exact form: warp e takes the words of packed lanes gq = e; its lanes spread over both column tiles, the two column
+        // halves, the four tq and the two row halves, so that one 8-byte store per lane covers two whole 128-byte rows of
+        // the swizzled tile (all 32 banks twice, no conflict).
+        // Dequantised form: a group has four warps, so warp e & 3 takes gq = 2*(e & 3) and 2*(e & 3) + 1 in turn.
+        const int x_ct2 = lane >> 4;
+        const int x_a = 2 * ((lane >> 3) & 1) + (lane & 1);
+        const int x_tq = (lane >> 1) & 3;
+        const int x_gq = DEQ ? 2 * (e & 3) : e;
+        const int x_l = 4 * x_gq + x_tq;
         const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
         const uint32_t x_aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
         int it = 0, tile_i = 0;
         for (int t = t_first; t < P.tile_hi; t += t_stride, ++tile_i) {
             const int rt = t / P.n_bt, bt = t % P.n_bt;
-            __half2 g_rows[kMaxPaths][8];                     // DEQ: output scales of this thread's eight rows, both halves alike
+            __half2 g_rows[kMaxPaths][2][8];                  // DEQ: output scales of this thread's 2 x 8 rows, both halves alike
             if (DEQ) {
 #pragma unroll
                 for (int k = 0; k < kMaxPaths; ++k)
 #pragma unroll
-                    for (int p = 0; p < 8; ++p) {
-                        const int r = rt * kTileM + 16 * p + x_gq + 8 * (x_a & 1);
-                        g_rows[k][p] = __half2half2((k < K && r < G.Mp) ? P.g[(size_t)k * G.Mp + r] : __float2half(0.f));
-                    }
+                    for (int gi = 0; gi < 2; ++gi)
+#pragma unroll
+                        for (int p = 0; p < 8; ++p) {
+                            const int r = rt * kTileM + 16 * p + x_gq + gi + 8 * (x_a & 1);
+                            g_rows[k][gi][p] = __half2half2((k < K && r < G.Mp) ? P.g[(size_t)k * G.Mp + r] : __float2half(0.f));
+                        }
             }
             for (int s = s_lo; s < s_hi; ++s, ++it) {
                 if (DEQ && (it & 1) != grp) continue;                 // the other group's step
@@ -315,23 +322,22 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                     // dequantised operand: for each of this thread's 8 rows and 4 columns, sum_k +-g_k[row] h_k[col],
                     // accumulated from the last (smallest) path to the first with one fused multiply-add per path
 #pragma unroll
-                    for (int ct2 = 0; ct2 < 2; ++ct2) {
-                        if (ct2 >= cts) break;
+                    for (int gi = 0; gi < 2; ++gi) {
+                        const int gq = x_gq + gi, l = x_l + 4 * gi;
                         uint32_t u01[kMaxPaths], u23[kMaxPaths];
                         uint2 hv[kMaxPaths];
 #pragma unroll
                         for (int k = 0; k < kMaxPaths; ++k) {
                             uint32_t w = 0;
                             hv[k] = make_uint2(0u, 0u);
-                            if (k < K) {
-                                w = reinterpret_cast<const uint32_t*>(&st.bits[k][ct2][x_l])[x_a];
-                                hv[k] = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff + 32 * ct2]);
+                            if (k < K && x_ct2 < cts) {
+                                w = reinterpret_cast<const uint32_t*>(&st.bits[k][x_ct2][l])[x_a];
+                                hv[k] = *reinterpret_cast<const uint2*>(&st.h[k][x_hoff]);
                             }
                             u01[k] = __byte_perm(w, 0u, 0x1404);
                             u23[k] = __byte_perm(w, 0u, 0x3424);
                         }
-                        // the 16-byte chunk index of the row gains 4 per column tile before the XOR swizzle
-                        const uint32_t aoff = (uint32_t)((x_gq + 8 * (x_a & 1)) * 128 + (((4 * ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ x_gq) << 4) + 8 * (x_tq & 1));
+                        const uint32_t aoff = (uint32_t)((gq + 8 * (x_a & 1)) * 128 + (((4 * x_ct2 + 2 * (x_a >> 1) + (x_tq >> 1)) ^ gq) << 4) + 8 * (x_tq & 1));
                         const uint32_t dst = smem_u32(ast.a[0]) + aoff;
 #pragma unroll
                         for (int p = 0; p < 8; ++p) {
@@ -341,8 +347,8 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
                                 if (k >= K) continue;
                                 const uint32_t ox = hv[k].x ^ ((u01[k] << (7 - p)) & 0x80008000u);   // +-h: sign flipped where the weight is -1
                                 const uint32_t oy = hv[k].y ^ ((u23[k] << (7 - p)) & 0x80008000u);
-                                s01 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&ox), s01);
-                                s23 = __hfma2(g_rows[k][p], *reinterpret_cast<const __half2*>(&oy), s23);
+                                s01 = __hfma2(g_rows[k][gi][p], *reinterpret_cast<const __half2*>(&ox), s01);
+                                s23 = __hfma2(g_rows[k][gi][p], *reinterpret_cast<const __half2*>(&oy), s23);
                             }
                             asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + p * 16 * 128), "r"(*reinterpret_cast<const uint32_t*>(&s01)),
                                          "r"(*reinterpret_cast<const uint32_t*>(&s23)) : "memory");
