@@ -111,8 +111,10 @@ RABIT_API int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uin
  *   x  DEVICE fp16 [batch][N] row-major, 16-byte aligned
  *   y  DEVICE fp16 [batch][M] row-major, 16-byte aligned, must not overlap x
  * Asynchronous on `stream`; allocates nothing, never synchronises, and may be captured in
- * a CUDA graph.  batch <= 16 runs the bandwidth-bound GEMV family, larger batches the
- * tensor-core GEMM.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end.
+ * a CUDA graph.  Up to 4 batch rows run the bandwidth-bound GEMV (one pass over the weights), more
+ * than 16 the tensor-core GEMM; in between, GEMV passes of four rows or one GEMM launch, whichever the
+ * library's cost estimate for this shape favours.  A GEMM with few output tiles runs as clusters of CTAs
+ * that share a tile's contraction.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end.
  */
 RABIT_API int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
