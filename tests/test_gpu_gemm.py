@@ -129,6 +129,7 @@ def test_dequantised_tile_gemm(K, M, N, batch):
     (2, 1024, 8192, 512, GEMM),    # the 70B k/v projection at batch 512: 16 tiles, eight CTAs each
     (2, 19200, 1024, 20, GEMM),    # 150 tiles on 148 SMs: one whole wave, then the two tiles left over as a split launch
     (2, 19100, 1024, 20, DEQ),
+    (2, 11008, 1024, 40, GEMM),    # 86 tiles: more than half the SMs, one CTA per tile
 ])
 def test_gemm_split_contraction_across_a_cluster(K, M, N, batch, variant):
     """Layers with few output tiles: the CTAs of a cluster split the contraction of a tile and add their partial
