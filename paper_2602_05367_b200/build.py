@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librabit.so")
-SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemm_tc.cu",
+SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemv_lut.cu", "rabit_gemm_tc.cu",
            "rabit_noalloc.cu", "rabit_derive.cu", "rabit_selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

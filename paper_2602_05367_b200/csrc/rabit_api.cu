@@ -20,6 +20,24 @@ void rabit_clear_error() { g_err[0] = 0; }
 
 extern "C" const char* rabit_last_error(void) { return g_err; }
 
+static void bind_layer(rabit_layer* L, const RabitGeom& G, const RabitHeader& hdr, void* dev_buf, int device) {
+    L->geom = G;
+    L->device = device;
+    L->variant = 0;
+    L->sm_count = 0;
+    cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, device);
+    L->dev_base = (char*)dev_buf;
+    L->dev_bytes = hdr.total_bytes;
+    L->d_bits = (const uint4*)(L->dev_base + hdr.off_bits);
+    L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
+    L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
+    L->d_partial = (float*)(L->dev_base + hdr.off_partial);
+    L->d_flags = (unsigned int*)(L->dev_base + hdr.off_flags);
+    L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
+    L->d_lut = (const unsigned char*)(L->dev_base + hdr.off_lut);
+    L->d_acc = (unsigned long long*)(L->dev_base + hdr.off_acc);
+}
+
 extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
                           int K, int M, int N, void* dev_buf, size_t dev_bytes, void* stream,
                           rabit_layer** out) {
@@ -57,43 +75,18 @@ extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint1
     if (!L) return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: out of host memory");
     RabitHeader packed_hdr;
     std::memcpy(&packed_hdr, image.data(), sizeof(packed_hdr));
-    if (!rabit_geom_from_header(packed_hdr, &L->geom)) {
+    RabitGeom packed_geom;
+    if (!rabit_geom_from_header(packed_hdr, &packed_geom)) {
         delete L;
         return rabit_fail(RABIT_INVALID_ARG, "rabit_pack: internal error, packed header unreadable");
     }
-    L->device = attr.device;
-    L->variant = 0;
-    L->sm_count = 0;
-    cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, attr.device);
-    L->dev_base = (char*)dev_buf;
-    L->dev_bytes = hdr.total_bytes;
-    L->d_bits = (const uint4*)(L->dev_base + hdr.off_bits);
-    L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
-    L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
-    L->d_partial = (float*)(L->dev_base + hdr.off_partial);
-    L->d_flags = (unsigned int*)(L->dev_base + hdr.off_flags);
-    L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
+    bind_layer(L, packed_geom, packed_hdr, dev_buf, attr.device);
     *out = L;
     return RABIT_OK;
 }
 
 static bool ranges_overlap(const void* a, size_t an, const void* b, size_t bn);
 
-static void bind_layer(rabit_layer* L, const RabitGeom& G, const RabitHeader& hdr, void* dev_buf, int device) {
-    L->geom = G;
-    L->device = device;
-    L->variant = 0;
-    L->sm_count = 0;
-    cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, device);
-    L->dev_base = (char*)dev_buf;
-    L->dev_bytes = hdr.total_bytes;
-    L->d_bits = (const uint4*)(L->dev_base + hdr.off_bits);
-    L->d_g = (const uint16_t*)(L->dev_base + hdr.off_g);
-    L->d_h = (const uint16_t*)(L->dev_base + hdr.off_h);
-    L->d_partial = (float*)(L->dev_base + hdr.off_partial);
-    L->d_flags = (unsigned int*)(L->dev_base + hdr.off_flags);
-    L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
-}
 
 extern "C" int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uint16_t* h, int K, int M, int N,
                                  void* dev_buf, size_t dev_bytes, void* stream, rabit_layer** out) {
@@ -126,10 +119,16 @@ extern "C" int rabit_derive_pack(const float* W_dev, const uint16_t* g, const ui
     // scales from the host (a few KB), the scratch sections by device-side fills
     RABIT_CUDA_TRY(cudaMemcpyAsync(base + hdr.off_g, tail.data(), tail.size(), cudaMemcpyHostToDevice, st));
     RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_partial, 0xFF, (size_t)(hdr.off_flags - hdr.off_partial), st));
-    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_flags, 0, (size_t)(hdr.total_bytes - hdr.off_flags), st));
+    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_flags, 0, (size_t)(hdr.off_lut - hdr.off_flags), st));
     cudaError_t e = rabit_launch_derive(G, W_dev, (const uint16_t*)(base + hdr.off_g), (const uint16_t*)(base + hdr.off_h),
                                         (uint4*)(base + hdr.off_bits), st);
+    if (e == cudaSuccess) e = rabit_launch_tiles_to_lut(G, (const uint4*)(base + hdr.off_bits), (unsigned char*)(base + hdr.off_lut), st);
     if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_derive_pack: launch failed: %s", cudaGetErrorString(e));
+    // The accumulate words are cleared AFTER the kernels on purpose: the decode kernels start copying weights before
+    // they wait for the previous kernel in the stream (weights normally never depend on it).  A fill between the
+    // kernels that write this layer's weights and its first use is an ordinary stream dependency, which such a
+    // kernel cannot overtake.
+    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_acc, 0, (size_t)(hdr.total_bytes - hdr.off_acc), st));
     // No synchronisation: copies from pageable host memory return once the source has been staged, so the
     // local buffers may go out of scope; the layer is usable by later work on the same stream.
     rabit_layer* L = new (std::nothrow) rabit_layer;
@@ -155,10 +154,18 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
     if (ranges_overlap(x, (size_t)batch * G.N * 2, y, (size_t)batch * G.M * 2))
         return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: x and y overlap");
     cudaStream_t st = (cudaStream_t)stream;
+    {
+        int dev = -1;
+        RABIT_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev != layer->device)
+            return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: the layer lives on device %d but device %d is current", layer->device, dev);
+    }
 
     int variant = layer->variant;
     if (variant == 0) {
-        if (batch <= RABIT_MAX_GEMV_BATCH) {
+        if (rabit_gemv_lut_supports(*layer, batch)) {
+            variant = 5;
+        } else if (batch <= RABIT_MAX_GEMV_BATCH) {
             variant = rabit_gemv_mma_supports(*layer, batch) ? 2 : 1;
             // From 5 batch rows on the GEMV makes two to four passes over the weights; the tensor-core GEMM, whose cost
             // does not depend on the batch up to 256, is then often cheaper.  Both estimates are fits to measurements
@@ -194,6 +201,16 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
                 return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: tcgen05 GEMM cannot run batch %d", batch);
             e = rabit_launch_gemm_tc(*layer, x, y, batch, st, true);
             break;
+        case 5: {
+            if (!rabit_gemv_lut_supports(*layer, 1))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: table-driven GEMV cannot run this layer");
+            const int rows = rabit_gemv_lut_supports(*layer, rabit_gemv_lut_max_rows()) ? rabit_gemv_lut_max_rows() : 1;
+            e = cudaSuccess;
+            for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += rows)             // up to `rows` batch rows share one pass over the weights
+                e = rabit_launch_gemv_lut(*layer, (const char*)x + (size_t)b0 * G.N * 2, (char*)y + (size_t)b0 * G.M * 2,
+                                          batch - b0 >= rows ? rows : batch - b0, st);
+            break;
+        }
         default:
             e = rabit_launch_plain(*layer, x, y, batch, st);
             break;
@@ -225,6 +242,30 @@ extern "C" int rabit_linear_group(const rabit_layer* const* layers, const void* 
         }
     }
     cudaStream_t st = (cudaStream_t)stream;
+    {
+        int dev = -1;
+        RABIT_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev != layers[0]->device)
+            return rabit_fail(RABIT_INVALID_ARG, "rabit_linear_group: the layers live on device %d but device %d is current", layers[0]->device, dev);
+    }
+    {
+        bool lut = rabit_gemv_lut_group_supports(layers, n_layers, batch);
+        for (int l = 0; l < n_layers && lut; ++l) lut = layers[l]->variant == 0 || layers[l]->variant == 5;
+        if (lut) {
+            cudaError_t e = rabit_launch_gemv_lut_group(layers, n_layers, xs, ys, batch, st, nullptr, nullptr);
+            if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear_group: launch failed: %s", cudaGetErrorString(e));
+            return RABIT_OK;
+        }
+    }
+    for (int a = 0; a < n_layers; ++a)
+        for (int b = a + 1; b < n_layers; ++b)
+            if (layers[a] == layers[b]) {                        // the same layer twice would share one reduction scratch: no fused launch
+                for (int l = 0; l < n_layers; ++l) {
+                    int rc = rabit_linear(layers[l], xs[l], ys[l], batch, stream);
+                    if (rc != RABIT_OK) return rc;
+                }
+                return RABIT_OK;
+            }
     bool fused = rabit_gemv_mma_group_supports(layers, n_layers, batch);
     for (int l = 0; l < n_layers && fused; ++l) fused = layers[l]->variant == 0 || layers[l]->variant == 2;
     if (!fused) {
@@ -383,7 +424,7 @@ extern "C" int rabit_layer_N(const rabit_layer* layer) { return layer ? layer->g
 extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
-    if (variant < 0 || variant > 4) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..4");
+    if (variant < 0 || variant > 5) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..5");
     layer->variant = variant;
     return RABIT_OK;
 }

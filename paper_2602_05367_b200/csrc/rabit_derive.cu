@@ -82,7 +82,55 @@ rabit_derive_kernel(RabitGeom G, const float* __restrict__ W, const __half* __re
     }
 }
 
+// Second arrangement of the same signs: the look-up blocks (rabit_layout.h), gathered from the tiles that the
+// kernel above has just written.  One warp per (path, row block of 32 rows, slice of 256 columns) = one 1 KB part;
+// lane = row.  A byte of eight consecutive columns comes from two tile words (four columns each, the row's bit p
+// in every byte).  Columns beyond N stay zero.
+__global__ void __launch_bounds__(kWarps * 32)
+rabit_tiles_to_lut_kernel(RabitGeom G, const uint32_t* __restrict__ tiles, uint4* __restrict__ lut) {
+    const int lane = threadIdx.x & 31;
+    const long long wid = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const long long parts = (long long)G.n_cs * G.n_rb * G.K;
+    if (wid >= parts) return;
+    const int k = (int)(wid % G.K);
+    const long long pos = wid / G.K;
+    const int rb = (int)(pos % G.n_rb), cs = (int)(pos / G.n_rb);
+    const int row = rb * RABIT_LUT_ROWS + lane;
+    const int rt = row >> 7, rl = row & 127, p = rl >> 4, gq = rl & 7, alo = (rl >> 3) & 1;
+    uint32_t out[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out[j] = 0u;
+#pragma unroll 4
+    for (int s = 0; s < 32; ++s) {
+        const int group = (s + lane) & 31;                              // byte group of the slice this lane stores at step s
+        const int col = cs * RABIT_LUT_COLS + 8 * group;
+        uint32_t byte = 0u;
+        if (col < G.N) {
+            const int ct = col >> 5, cl = col & 31, ah = cl >> 4, tq0 = (cl & 15) >> 2;     // tq0 is 0 or 2
+            const uint32_t* tile = tiles + rabit_tile_pos(G, rt, k, ct) * (RABIT_TILE_BYTES / 4);
+            const int a = alo | (ah << 1);
+            const uint32_t w0 = tile[(4 * gq + tq0) * 4 + a], w1 = tile[(4 * gq + tq0 + 1) * 4 + a];
+            const uint32_t n0 = ((((w0 >> p) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;  // bit c <- byte c
+            const uint32_t n1 = ((((w1 >> p) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;
+            byte = n0 | (n1 << 4);
+        }
+        out[s >> 2] |= byte << (8 * (s & 3));
+    }
+    uint4* dst = lut + (size_t)wid * (RABIT_LUT_PART_BYTES / 16);
+    dst[lane] = make_uint4(out[0], out[1], out[2], out[3]);
+    dst[32 + lane] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
 }  // namespace
+
+cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, cudaStream_t stream) {
+    const long long warps = (long long)G.n_cs * G.n_rb * G.K;
+    const long long blocks = (warps + kWarps - 1) / kWarps;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    rabit_tiles_to_lut_kernel<<<(unsigned int)blocks, kWarps * 32, 0, stream>>>(G, reinterpret_cast<const uint32_t*>(d_tiles),
+                                                                               reinterpret_cast<uint4*>(d_lut));
+    return cudaGetLastError();
+}
 
 cudaError_t rabit_launch_derive(const RabitGeom& G, const float* W, const uint16_t* d_g, const uint16_t* d_h, uint4* d_tiles,
                                 cudaStream_t stream) {

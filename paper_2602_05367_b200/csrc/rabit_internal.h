@@ -12,7 +12,7 @@
 struct rabit_layer {
     RabitGeom geom;
     int device;
-    int variant;                 // 0 auto, 1 plain, 2 integer-MMA GEMV, 3 tcgen05 GEMM
+    int variant;                 // 0 auto, 1 plain, 2 integer-MMA GEMV, 3 tcgen05 GEMM, 4 dequantised-tile GEMM, 5 table-driven GEMV
     int sm_count;
     char* dev_base;              // caller-owned packed image
     size_t dev_bytes;
@@ -22,6 +22,8 @@ struct rabit_layer {
     float* d_partial;            // fp32 [n_rt*K + RABIT_MAX_GRID][RABIT_PARTIAL_BATCH][128] cross-CTA partial sums (all-ones words between calls)
     unsigned int* d_flags;       // u32 [n_rt*K + RABIT_MAX_GRID] reserved (zero), then one status word
     unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
+    const unsigned char* d_lut;  // look-up blocks (table-driven GEMV)
+    unsigned long long* d_acc;   // u64 [RABIT_LUT_MAX_BATCH][Mp] accumulate words of the table-driven GEMV (zero between calls)
 };
 
 // error reporting (thread-local message); returns `code`
@@ -38,6 +40,7 @@ void rabit_clear_error();
 bool rabit_make_geom(int K, int M, int N, RabitGeom* out);          // hmax left at 0
 void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr);
 bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out); // validates magic, version and shape
+void rabit_scale_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* G);   // hmax and the fixed-point grid
 
 // header + scale sections, for images whose tiles are written on the device (rabit_pack.cu)
 #ifdef __cplusplus
@@ -48,6 +51,8 @@ bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N,
 cudaError_t rabit_launch_derive(const RabitGeom& G, const float* W, const uint16_t* d_g, const uint16_t* d_h, uint4* d_tiles,
                                 cudaStream_t stream);
 
+cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, cudaStream_t stream);
+
 // kernel launchers; each enqueues on `stream` and returns a cudaError_t from the launch
 cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
@@ -57,6 +62,13 @@ int rabit_gemv_mma_max_rows();
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream);
+// table-driven GEMV (rabit_gemv_lut.cu); acc_override / status_override redirect the scratch (nullptr: the image's own)
+cudaError_t rabit_launch_gemv_lut(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+bool rabit_gemv_lut_supports(const rabit_layer& L, int batch);
+int rabit_gemv_lut_max_rows();
+bool rabit_gemv_lut_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
+cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
+                                        int batch, cudaStream_t stream, unsigned long long* const* acc_override, unsigned int* status_override);
 cudaError_t rabit_launch_gemm_tc(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream, bool dequantised = false);
 bool rabit_gemm_tc_supports(const rabit_layer& L, int batch);
 double rabit_gemm_tc_estimate_us(const rabit_layer& L, int batch);

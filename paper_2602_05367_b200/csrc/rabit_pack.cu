@@ -36,8 +36,57 @@ bool rabit_make_geom(int K, int M, int N, RabitGeom* out) {
     G.n_rt = G.Mp / RABIT_TILE_ROWS;
     G.n_ct = N / RABIT_TILE_COLS;
     for (int k = 0; k < RABIT_MAX_K; ++k) G.hmax[k] = 0.f;
+    G.n_rb = G.Mp / RABIT_LUT_ROWS;
+    G.n_cs = (N + RABIT_LUT_COLS - 1) / RABIT_LUT_COLS;
+    G.fix_bits = 0;
+    G.unit_exp = 0;
     *out = G;
     return true;
+}
+
+// Everything the header records about the scales: max_j |h_k[j]| per path (the integer-MMA GEMV derives its
+// fixed-point scale from it) and the fixed-point grid of the table-driven GEMV's accumulate words.
+//
+// That GEMV adds, per output row, one partial sum per 256-column slice into a 64-bit word with an integer
+// atomic.  A partial sum is bounded, for ANY finite fp16 activations, by
+//     65504 * max_i sum_k |g_k[i]| * max_{k, slice} sum_{j in slice} |h_k[j]|,
+// so a grid of 2^unit_exp whose 2^fix_bits steps cover twice that bound can never overflow, and with
+// fix_bits = 54 - ceil(log2(slices)) the sum of all slices (each shifted to be non-negative) stays below 2^55.
+void rabit_scale_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* G) {
+    for (int k = 0; k < K; ++k) {
+        float m = 0.f;
+        for (int j = 0; j < N; ++j) {
+            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
+            if (m == m && (v > m || v != v)) m = v;   // a NaN scale makes the bound NaN
+        }
+        G->hmax[k] = m;
+    }
+    double gsum_max = 0.0;
+    for (int i = 0; i < M; ++i) {
+        double s = 0.0;
+        for (int k = 0; k < K; ++k) s += std::fabs((double)half_bits_to_float(g[(size_t)k * M + i]));
+        if (s > gsum_max || s != s) gsum_max = s;
+    }
+    double hsum_max = 0.0;
+    for (int k = 0; k < K; ++k)
+        for (int j0 = 0; j0 < N; j0 += RABIT_LUT_COLS) {
+            double s = 0.0;
+            for (int j = j0; j < N && j < j0 + RABIT_LUT_COLS; ++j) s += std::fabs((double)half_bits_to_float(h[(size_t)k * N + j]));
+            if (s > hsum_max || s != s) hsum_max = s;
+        }
+    int clog = 0;
+    while ((1 << clog) < G->n_cs) ++clog;
+    G->fix_bits = 54 - clog;
+    const double bound = 65504.0 * gsum_max * hsum_max;
+    int e = 0;
+    if (bound == bound && bound > 0.0 && bound < 1e300) {
+        int ex = 0;
+        std::frexp(bound, &ex);                       // bound < 2^ex
+        e = ex + 1;                                   // one spare bit for the fp32 roundings of the kernel
+    }
+    if (e < -40) e = -40;                             // keeps 2^(fix_bits - e) inside fp32
+    if (e > 100) e = 100;
+    G->unit_exp = e - G->fix_bits;
 }
 
 void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr) {
@@ -49,12 +98,16 @@ void rabit_fill_header(const RabitGeom& G, RabitHeader* hdr) {
     hdr->max_grid = RABIT_MAX_GRID;
     hdr->partial_batch = RABIT_PARTIAL_BATCH;
     for (int k = 0; k < G.K; ++k) std::memcpy(&hdr->hmax_bits[k], &G.hmax[k], 4);
+    hdr->n_rb = G.n_rb; hdr->n_cs = G.n_cs;
+    hdr->fix_bits = (uint32_t)G.fix_bits; hdr->unit_exp = G.unit_exp;
     size_t off = RABIT_HEADER_BYTES;
     hdr->off_bits = off;     off = rabit_align256(off + (size_t)G.K * G.n_rt * G.n_ct * RABIT_TILE_BYTES);
     hdr->off_g = off;        off = rabit_align256(off + (size_t)G.K * G.Mp * 2);
     hdr->off_h = off;        off = rabit_align256(off + (size_t)G.K * G.N * 2);
     hdr->off_partial = off;  off = rabit_align256(off + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID) * RABIT_PARTIAL_BATCH * RABIT_TILE_ROWS * 4);
     hdr->off_flags = off;    off = rabit_align256(off + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID) * 4 + 4);   // + one status word
+    hdr->off_lut = off;      off = rabit_align256(off + (size_t)G.n_cs * G.n_rb * G.K * RABIT_LUT_PART_BYTES);
+    hdr->off_acc = off;      off = rabit_align256(off + (size_t)RABIT_LUT_MAX_BATCH * G.Mp * 8);
     hdr->total_bytes = off;
 }
 
@@ -63,6 +116,9 @@ bool rabit_geom_from_header(const RabitHeader& hdr, RabitGeom* out) {
     if (!rabit_make_geom((int)hdr.K, (int)hdr.M, (int)hdr.N, out)) return false;
     if (hdr.max_grid != RABIT_MAX_GRID || hdr.partial_batch != RABIT_PARTIAL_BATCH) return false;
     for (int k = 0; k < out->K; ++k) std::memcpy(&out->hmax[k], &hdr.hmax_bits[k], 4);
+    if (hdr.n_rb != (uint32_t)out->n_rb || hdr.n_cs != (uint32_t)out->n_cs) return false;
+    out->fix_bits = (int)hdr.fix_bits;
+    out->unit_exp = hdr.unit_exp;
     return true;
 }
 
@@ -110,14 +166,7 @@ bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N,
                       std::vector<uint8_t>* tail) {
     RabitGeom G;
     if (!rabit_make_geom(K, M, N, &G)) return false;
-    for (int k = 0; k < K; ++k) {
-        float m = 0.f;
-        for (int j = 0; j < N; ++j) {
-            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
-            if (m == m && (v > m || v != v)) m = v;
-        }
-        G.hmax[k] = m;
-    }
+    rabit_scale_meta(g, h, K, M, N, &G);
     rabit_fill_header(G, hdr);
     tail->assign((size_t)(hdr->off_partial - hdr->off_g), 0);
     uint8_t* base = tail->data() - hdr->off_g;                    // so that image offsets can be used
@@ -138,14 +187,7 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
     RabitGeom G;
     if (!rabit_make_geom(K, M, N, &G))
         return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_pack_host: unsupported shape K=%d M=%d N=%d (need 1<=K<=3, M>=1, N%%32==0)", K, M, N);
-    for (int k = 0; k < K; ++k) {
-        float m = 0.f;
-        for (int j = 0; j < N; ++j) {
-            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
-            if (m == m && (v > m || v != v)) m = v;   // a NaN scale makes the bound NaN
-        }
-        G.hmax[k] = m;
-    }
+    rabit_scale_meta(g, h, K, M, N, &G);
     RabitHeader hdr;
     rabit_fill_header(G, &hdr);
     if (out_bytes < hdr.total_bytes)
@@ -166,11 +208,25 @@ extern "C" int rabit_pack_host(const uint32_t* planes, const uint16_t* g, const 
                     pack_tile(G, planes + (size_t)k * plane_words, rt, ct,
                               bits + rabit_tile_pos(G, rt, k, ct) * RABIT_TILE_BYTES);
     };
+    // look-up blocks: the canonical bytes (eight consecutive columns of one row), permuted
+    uint8_t* lut = base + hdr.off_lut;
+    const int row_bytes = N / 8;
+    auto work_lut = [&](int tid) {
+        for (int k = 0; k < K; ++k)
+            for (int row = tid; row < M; row += nthreads) {
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(planes + (size_t)k * plane_words + (size_t)row * (N / 32));
+                for (int cb = 0; cb < row_bytes; ++cb) lut[rabit_lut_byte_offset(G, k, row, cb)] = src[cb];
+            }
+    };
     if (nthreads == 1) {
         work(0);
+        work_lut(0);
     } else {
         std::vector<std::thread> pool;
         for (int t = 0; t < nthreads; ++t) pool.emplace_back(work, t);
+        for (auto& th : pool) th.join();
+        pool.clear();
+        for (int t = 0; t < nthreads; ++t) pool.emplace_back(work_lut, t);
         for (auto& th : pool) th.join();
     }
     uint16_t* gp = (uint16_t*)(base + hdr.off_g);
@@ -217,6 +273,18 @@ extern "C" int rabit_unpack_host(const void* image, size_t image_bytes,
                                 }
                             }
                 }
+    }
+    if (planes_out) {
+        // the look-up blocks must describe the same signs as the tiles
+        const uint8_t* lut = base + hdr.off_lut;
+        for (int k = 0; k < K; ++k)
+            for (int row = 0; row < M; ++row) {
+                const uint8_t* want = reinterpret_cast<const uint8_t*>(planes_out + ((size_t)k * M + row) * words_per_row);
+                for (int cb = 0; cb < N / 8; ++cb)
+                    if (lut[rabit_lut_byte_offset(G, k, row, cb)] != want[cb])
+                        return rabit_fail(RABIT_INVALID_ARG, "rabit_unpack_host: the tile section and the look-up section disagree (path %d, row %d, columns %d..%d)",
+                                          k, row, 8 * cb, 8 * cb + 7);
+            }
     }
     const uint16_t* gp = (const uint16_t*)(base + hdr.off_g);
     const uint16_t* hp = (const uint16_t*)(base + hdr.off_h);

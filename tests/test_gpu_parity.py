@@ -12,7 +12,7 @@ from tests.gpu_util import run_layer, check_against_oracle
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [0, 1, 2]   # automatic, plain sign-select, integer-MMA GEMV
+VARIANTS = [0, 1, 2, 5]   # automatic, plain sign-select, integer-MMA GEMV, table-driven GEMV
 
 SMALL = [  # several tiles plus ragged tails in both dimensions
     (2, 32, 128), (2, 100, 160), (2, 256, 1184), (3, 96, 640), (1, 33, 96), (2, 160, 2080), (2, 1000, 512),

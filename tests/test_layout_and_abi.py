@@ -84,12 +84,66 @@ def test_single_bit_lands_where_the_definition_says():
     assert nz[0] == off and bits[off] == 1 << p
 
 
+def test_single_bit_lands_in_the_look_up_block_the_definition_names():
+    K, M, N = 2, 200, 544
+    L = make_layer(M, N, K, key=(87,))
+    for row, col, k in [(45, 203, 1), (0, 0, 0), (199, 543, 0), (31, 255, 1), (32, 256, 0), (77, 300, 1)]:
+        planes = make_planes_constant(K, M, N, 0)
+        planes[k, row, col // 32] = np.uint32(1 << (col % 32))
+        img = rabit.pack_host(planes, L.g, L.h)
+        hd = spec.read_header(img)
+        sec = img[hd["off_lut"]:hd["off_acc"]]
+        nz = np.flatnonzero(sec)
+        assert nz.size == 1
+        cs, cl = divmod(col, 256); group, b = divmod(cl, 8); rb, l = divmod(row, 32)
+        s = (group - l) % 32                                  # the step at which lane l visits this group
+        off = ((cs * hd["n_rb"] + rb) * K + k) * 1024 + 512 * (s // 16) + 16 * l + (s % 16)
+        assert nz[0] == off and sec[off] == 1 << b
+
+
+@pytest.mark.parametrize("K,M,N", [(2, 64, 256), (3, 33, 1056), (1, 7, 96), (2, 100, 160)])
+def test_look_up_blocks_alone_give_back_the_planes(K, M, N):
+    L = make_layer(M, N, K, key=(88, K, M, N))
+    img = rabit.pack_host(L.planes, L.g, L.h)
+    assert np.array_equal(spec.unpack_lut_spec(img), L.planes)
+    # an image whose two sign sections disagree is refused
+    hd = spec.read_header(img)
+    bad = img.copy()
+    bad[hd["off_lut"] + 16 * 3 + 1] ^= 0x10                  # (lane 3, step 1) of block 0, path 0: a column inside N for all shapes here
+    lib = binding.raw_lib()
+    planes = np.empty((K, M, N // 32), dtype=np.uint32)
+    assert lib.rabit_unpack_host(bad.ctypes.data, bad.nbytes, planes.ctypes.data, None, None) == -1
+    assert "disagree" in rabit.last_error()
+
+
+def test_header_records_the_fixed_point_grid():
+    """The grid must cover twice the largest possible partial sum of a slice: recomputed here from its definition."""
+    L = make_layer(96, 4096 + 256, 2, key=(89,))
+    hd = spec.read_header(rabit.pack_host(L.planes, L.g, L.h))
+    assert hd["n_cs"] == 17 and hd["fix_bits"] == 54 - 5
+    g = np.abs(L.g.astype(np.float64)); h = np.abs(L.h.astype(np.float64))
+    bound = 65504.0 * g.sum(axis=0).max() * max(h[k, j:j + 256].sum() for k in range(2) for j in range(0, h.shape[1], 256))
+    top = 2.0 ** (hd["unit_exp"] + hd["fix_bits"])
+    assert 2 * bound <= top < 8 * bound
+    # all-zero scales: any grid will do, the header holds e = 0
+    Z = make_layer(32, 64, 1, key=(90,))
+    hd = spec.read_header(rabit.pack_host(Z.planes, np.zeros_like(Z.g), Z.h))
+    assert hd["unit_exp"] == -hd["fix_bits"]
+
+
 def test_scratch_and_padding_are_zero():
     L = make_layer(40, 160, 2, key=(84,))
     img = rabit.pack_host(L.planes, L.g, L.h)
     hd = spec.read_header(img)
     assert (img[hd["off_partial"]:hd["off_flags"]] == 0xFF).all()       # resting state of the partial buffer
-    assert not img[hd["off_flags"]:hd["total_bytes"]].any()
+    assert not img[hd["off_flags"]:hd["off_lut"]].any()
+    assert not img[hd["off_acc"]:hd["total_bytes"]].any()               # accumulate words rest at zero
+    # look-up blocks: rows beyond M and columns beyond N hold bit 0 (160 columns -> one slice of 256)
+    lut = img[hd["off_lut"]:hd["off_acc"]][:hd["n_cs"] * hd["n_rb"] * 2 * 1024].reshape(hd["n_cs"], hd["n_rb"], 2, 2, 32, 16)
+    hf, l, q = np.meshgrid(np.arange(2), np.arange(32), np.arange(16), indexing="ij")
+    group = (16 * hf + q + l) % 32
+    assert not lut[:, :, :, group >= 160 // 8].any()
+    assert not lut[:, 1, :, :, 8:, :].any() and not lut[:, 2:].any()    # rows 40..63, then whole padded row blocks
     g = img[hd["off_g"]:hd["off_h"]].view(np.uint16)[:2 * hd["Mp"]].reshape(2, hd["Mp"])
     assert not g[:, 40:].any()
 
