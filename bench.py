@@ -119,7 +119,7 @@ def whole_job_us_per_layer(ms_per_step: float, layers_per_step: int, world: int)
 # ---------------------------------------------------------------------------------------
 # workload
 # ---------------------------------------------------------------------------------------
-def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: int = 1):
+def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: int = 1, hints: bool = True):
     import torch
     import paper_2602_05367_b200 as rabit
     from synth import llama2_7b_layer_shapes, make_layer, make_x
@@ -132,6 +132,17 @@ def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: 
             L = make_layer(sh.M, sh.N, K_PATHS, key=(seed_cfg, c, p))
             row.append(rabit.rabit_pack(L.planes, L.g, L.h, device=device))
         layers.append(row)
+    if hints:
+        # the order a decoder runs them in: q|k|v -> o -> gate|up -> down -> the next decoder layer's q|k|v
+        for c in range(copies):
+            nxt = layers[(c + 1) % copies]
+            row = layers[c]
+            for p in (0, 1, 2):
+                row[p].set_next([row[3]])
+            row[3].set_next([row[4], row[5]])
+            row[4].set_next([row[6]])
+            row[5].set_next([row[6]])
+            row[6].set_next([nxt[0], nxt[1], nxt[2]])
     widths = sorted({sh.N for sh in shapes})
     xs_host = {n: np.stack([make_x(batch, n, key=(seed_cfg, 10_000 + t)) for t in range(tokens)]) for n in widths}
     xs = {n: torch.from_numpy(a).to(device) for n, a in xs_host.items()}            # [tokens][batch][N]
@@ -183,7 +194,7 @@ def bench_rabit(args) -> dict:
         torch.cuda.synchronize()
 
     copies, batch, tokens = args.copies, args.batch, 16
-    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens)
+    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens, hints=not args.no_hints)
     step_bytes = sum(layer_bytes(sh.M, sh.N, batch) for sh in shapes)
     n_proj = len(shapes)
     stream = torch.cuda.Stream(device)
@@ -382,6 +393,8 @@ def bench_cases(args) -> dict:
     else:
         shapes, cfg = llama_70b_layer_shapes(), 4
         batches = [512] if args.workload == "gemm70b" else [1]
+    if args.only_shape:
+        shapes = [sh for sh in shapes if "%dx%d" % (sh.M, sh.N) == args.only_shape]
     peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     tc_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
@@ -533,6 +546,81 @@ def bench_derive(args) -> dict:
             "roofline": head["roofline"], "gpu_launches": len(cases) * 12}
 
 
+def bench_trace(args) -> dict:
+    """Extra workload: where the time of a decoder-layer step goes, from the phase stamps of a library built with
+    -DRABIT_TRACE (python paper_2602_05367_b200/build.py --trace; run with RABIT_LIBRARY=.../librabit_trace.so).
+    Three decoder layers (more than L2), one CUDA graph that walks them once, replayed; the stamps of the last
+    replay are reported per launch as microseconds after the entry of the cycle's first CTA (median over the CTAs of a
+    launch, and the latest CTA for the end stamps)."""
+    import ctypes
+    import torch
+    import paper_2602_05367_b200 as rabit
+    from paper_2602_05367_b200 import binding
+
+    torch.cuda.set_device(0)
+    device = "cuda:0"
+    copies = 3
+    shapes, layers, xs, xs_host, ys = build_workload(copies, 1, device, 16, hints=not args.no_hints)
+    lib = binding.raw_lib()
+    stream = torch.cuda.Stream(device)
+    grouped = not args.no_group
+    with torch.cuda.stream(stream):
+        for c in range(copies):
+            run_step(rabit, shapes, layers[c], xs, ys, c, grouped)
+    stream.synchronize()
+    buf = torch.zeros(1 << 22, dtype=torch.int64, device=device)
+    rc = lib.rabit_trace_begin(ctypes.c_void_p(buf.data_ptr()), buf.numel() * 8)
+    if rc != 0:
+        raise SystemExit("trace workload: " + rabit.last_error())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for c in range(copies):
+            run_step(rabit, shapes, layers[c], xs, ys, c, grouped)
+    n = lib.rabit_trace_launches(None, 0)
+    ctas = (ctypes.c_int * n)()
+    lib.rabit_trace_launches(ctas, n)
+    with torch.cuda.stream(stream):
+        for _ in range(20):
+            g.replay()
+    stream.synchronize()
+    lib.rabit_trace_begin(None, 0)
+    raw = buf.cpu().numpy().astype(np.uint64)
+    if args.trace_dump:
+        np.save(args.trace_dump, raw[:64 * int(sum(ctas))])
+        json.dump([int(c) for c in ctas], open(args.trace_dump + ".ctas.json", "w"))
+    names = ["entry", "wait_over", "x_arrived", "table_built", "first_weights", "last_lookup", "end", "first_block_done"]
+    mhz = 1965.0
+    rows, off, base = [], 0, None
+    for i in range(n):
+        full = raw[off:off + 64 * ctas[i]].reshape(ctas[i], 64).astype(np.float64)
+        rec = full[:, :8]
+        off += 64 * ctas[i]
+        if base is None:
+            base = rec[:, 0].min()
+        entry = (rec[:, 0] - base) / 1e3                                   # us, coarse
+        dur = rec[:, 1:] / mhz                                              # us since the CTA's entry (cycles / max SM clock)
+        row = {"launch": i, "ctas": int(ctas[i]), "entry_first": round(float(entry.min()), 2), "entry_med": round(float(np.median(entry)), 2),
+               "end_abs_max": round(float((entry + dur[:, 5]).max()), 2)}
+        for j, nm in enumerate(names[1:]):
+            row[nm + "_med"] = round(float(np.median(dur[:, j])), 3)
+            row[nm + "_max"] = round(float(dur[:, j].max()), 3)
+        rows.append(row)
+    sys.stderr.write("times in us; per launch: entry on the global timer (first CTA / median), the rest since each CTA's own entry (median / max over CTAs)\n")
+    sys.stderr.write("launch ctas | entry first   med | wait_over     | x_arrived     | table_built   | first_weights | first_blk_done| last_lookup   | end           | end(abs,max)\n")
+    for r in rows:
+        sys.stderr.write("%3d %4d | %7.2f %7.2f |" % (r["launch"], r["ctas"], r["entry_first"], r["entry_med"]))
+        for nm in ("wait_over", "x_arrived", "table_built", "first_weights", "first_block_done", "last_lookup", "end"):
+            sys.stderr.write(" %6.2f %6.2f |" % (r[nm + "_med"], r[nm + "_max"]))
+        sys.stderr.write(" %7.2f\n" % r["end_abs_max"])
+    for row in layers:
+        for L in row:
+            L.free()
+    return {"metric": "phase stamps of the decode GEMV launches (us after the first entry of the cycle)", "value": rows[-1]["end_abs_max"] / copies,
+            "unit": "us/step", "n_gpus": 1, "steps": copies, "warmup": 3, "ms_per_step": rows[-1]["end_abs_max"] / copies / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "trace7b", "copies": copies, "grouped": grouped}, "launches": rows, "gpu_launches": n}
+
+
 def bench_reference(args) -> dict:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -569,7 +657,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-group", action="store_true", help="one rabit_linear launch per projection (7 per step instead of 4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemm7b", "gemv70b", "sweep8b", "derive7b"],
+    ap.add_argument("--only-shape", default="", help="extra workloads: keep only the layer shape MxN (e.g. 28672x8192)")
+    ap.add_argument("--no-hints", action="store_true", help="do not tell the layers which layer runs next (no weight prefetch across launches)")
+    ap.add_argument("--trace-dump", default="", help="trace7b: also save the raw stamps (numpy file) here")
+    ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemm7b", "gemv70b", "sweep8b", "derive7b", "trace7b"],
                     help="decoder7b is the contract's line; the others are extra single-GPU measurements")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -578,6 +669,8 @@ def main():
         res = bench_reference(args)
     elif args.workload == "derive7b":
         res = bench_derive(args)
+    elif args.workload == "trace7b":
+        res = bench_trace(args)
     elif args.workload != "decoder7b":
         res = bench_cases(args)
     else:

@@ -206,6 +206,24 @@ RABIT_API size_t rabit_group_stage_bytes(const rabit_layer* const* layers, int n
 RABIT_API int rabit_linear_group_host(const rabit_layer* const* layers, const void* const* xs_host, void* const* ys_host,
                             int n_layers, int batch, void* dev_stage, size_t dev_stage_bytes, void* stream);
 
+/*
+ * Phase tracing of the decode kernels, for profiling (no counterpart in the paper).  Only a library built with
+ * -DRABIT_TRACE (python paper_2602_05367_b200/build.py --trace -> librabit_trace.so) records anything; in the
+ * ordinary build rabit_trace_begin returns RABIT_UNSUPPORTED_SHAPE and rabit_trace_launches 0.
+ *   rabit_trace_begin(dev_buf, bytes)  DEVICE buffer, 8-byte aligned, caller-owned; every later launch of the
+ *       table-driven GEMV (also launches captured into a CUDA graph from now on) gets the next record of
+ *       64 x uint64 per CTA in it until it is full; dev_buf = NULL stops tracing.  Not thread-safe.
+ *   rabit_trace_launches(ctas_out, max)  number of records handed out since rabit_trace_begin; ctas_out[i]
+ *       receives the CTA count of record i (records follow one another in the buffer).
+ * Stamps of a CTA, taken by one thread: 0 kernel entry in nanoseconds of the GPU's global timer (coarse: it advances
+ * in steps of a fraction of a microsecond); 1..7 SM clock cycles since that entry: 1 dependency wait over, 2 x and h
+ * of the first table have arrived, 3 first table built, 4 first weights in registers, 5 last look-up done and last
+ * atomic issued, 6 last atomic answered and y stored, 7 look-ups of the thread's first block answered; 8 + 5*i + {0..4}
+ * for the thread's block i < 11: loop top, weights arrived, look-ups answered, previous atomic settled, output scales arrived.
+ */
+RABIT_API int rabit_trace_begin(void* dev_buf, size_t bytes);
+RABIT_API int rabit_trace_launches(int* ctas_out, int max_launches);
+
 /* Copy the packed image back from the device and unpack it (round-trip check).  Synchronises. */
 RABIT_API int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint16_t* g_out, uint16_t* h_out,
                  void* stream);
@@ -225,6 +243,18 @@ RABIT_API int rabit_layer_N(const rabit_layer* layer);
  * Meant for A/B timing and profiling; results are within tolerance for every variant.
  */
 RABIT_API int rabit_set_variant(rabit_layer* layer, int variant);
+
+/*
+ * Prefetch hint for decode chains (no counterpart in the paper; the layer's result does not change).  Names up to 8
+ * layers that the caller will run right after `layer` (for a decoder: q|k|v -> o -> gate|up -> down -> the next
+ * block's q|k|v).  From then on the batch 1..2 kernel of `layer` (alone or inside a group) asks L2, at its very
+ * start, to fetch the look-up blocks of those layers, so that they cross HBM - and their pages enter the TLBs -
+ * while this kernel still waits for its input and computes, instead of at the start of their own kernel, which at
+ * a few microseconds per layer would otherwise begin with an idle HBM and a memory latency on its critical path.
+ * Every byte still crosses HBM once.  n_next = 0 removes the hint.  The device buffers of the named layers must
+ * stay allocated for as long as the hint is set (freeing their descriptors is fine; the hint keeps addresses).
+ */
+RABIT_API int rabit_set_next(rabit_layer* layer, const rabit_layer* const* next, int n_next);
 
 /* Release the descriptor only; the caller's device buffer is untouched. NULL is accepted. */
 RABIT_API int rabit_free(rabit_layer* layer);

@@ -9,7 +9,8 @@ from typing import Optional, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "librabit.so")
+# RABIT_LIBRARY selects another build of the same library (e.g. librabit_trace.so, built with --trace)
+_LIB_PATH = os.environ.get("RABIT_LIBRARY") or os.path.join(_HERE, "librabit.so")
 
 _c_void_p = ctypes.c_void_p
 _c_int = ctypes.c_int
@@ -66,8 +67,14 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = [_c_void_p]
     lib.rabit_set_variant.restype = _c_int
     lib.rabit_set_variant.argtypes = [_c_void_p, _c_int]
+    lib.rabit_set_next.restype = _c_int
+    lib.rabit_set_next.argtypes = [_c_void_p, _c_void_p, _c_int]
     lib.rabit_free.restype = _c_int
     lib.rabit_free.argtypes = [_c_void_p]
+    lib.rabit_trace_begin.restype = _c_int
+    lib.rabit_trace_begin.argtypes = [_c_void_p, _c_size_t]
+    lib.rabit_trace_launches.restype = _c_int
+    lib.rabit_trace_launches.argtypes = [_c_void_p, _c_int]
     lib.rabit_last_error.restype = ctypes.c_char_p
     return lib
 
@@ -152,8 +159,17 @@ class RabitLayer:
 
     def set_variant(self, variant: int) -> None:
         """Kernel family for later rabit_linear calls of this layer: 0 automatic, 1 plain, 2 integer tensor-core GEMV,
-        3 tcgen05 GEMM (exact expansion), 4 tcgen05 GEMM on dequantised fp16 weight tiles (never chosen automatically)."""
+        3 tcgen05 GEMM (exact expansion), 4 tcgen05 GEMM on dequantised fp16 weight tiles (never chosen automatically),
+        5 table-driven GEMV."""
         _check(_lib.rabit_set_variant(self.handle, variant))
+
+    def set_next(self, next_layers) -> None:
+        """Prefetch hint: the layers that will run right after this one (up to 8; an empty list removes the hint).
+        The named layers' device buffers must stay alive while the hint is set."""
+        n = len(next_layers)
+        arr = (_c_void_p * max(n, 1))(*[l.handle for l in next_layers])
+        _check(_lib.rabit_set_next(self.handle, arr, n))
+        self._next_keepalive = [l.dev_buf for l in next_layers]
 
     def status(self, clear: bool = False, stream: int = 0) -> int:
         """0 if every kernel of this layer completed its waits, RABIT_DEVICE_FAULT (-5) otherwise; synchronises."""
@@ -172,6 +188,7 @@ class RabitLayer:
             self._handle = None
             self.dev_buf = None
             self._stage = None
+            self._next_keepalive = None
 
     def __del__(self):  # pragma: no cover
         try:

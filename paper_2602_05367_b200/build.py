@@ -12,6 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librabit.so")
+LIB_TRACE = os.path.join(HERE, "librabit_trace.so")          # the same sources with -DRABIT_TRACE (phase stamps)
 SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemv_lut.cu", "rabit_gemm_tc.cu",
            "rabit_noalloc.cu", "rabit_derive.cu", "rabit_selftest.cu"]
 NVCC_FLAGS = [
@@ -33,18 +34,19 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    if not trace and not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + _sources()
+    out = LIB_TRACE if trace else LIB
+    cmd = [nvcc] + NVCC_FLAGS + (["-DRABIT_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else []) + ["-o", out] + _sources()
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode != 0:
         sys.stderr.write(proc.stdout + proc.stderr)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed building librabit.so")
-    return LIB
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, trace="--trace" in sys.argv))

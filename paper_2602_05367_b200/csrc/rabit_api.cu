@@ -36,6 +36,7 @@ static void bind_layer(rabit_layer* L, const RabitGeom& G, const RabitHeader& hd
     L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
     L->d_lut = (const unsigned char*)(L->dev_base + hdr.off_lut);
     L->d_acc = (unsigned long long*)(L->dev_base + hdr.off_acc);
+    L->n_next = 0;
 }
 
 extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
@@ -417,6 +418,55 @@ extern "C" int rabit_unpack(const rabit_layer* layer, uint32_t* planes_out, uint
     return rabit_unpack_host(image.data(), image.size(), planes_out, g_out, h_out);
 }
 
+// ---- phase tracing (only does something in a library built with -DRABIT_TRACE) -------------------
+#ifdef RABIT_TRACE
+static unsigned long long* g_trace_buf = nullptr;
+static size_t g_trace_words = 0, g_trace_used = 0;
+static std::vector<int> g_trace_ctas;                                    // CTAs of every traced launch, in launch order
+#endif
+
+unsigned long long* rabit_trace_slot(int ctas) {
+#ifdef RABIT_TRACE
+    if (!g_trace_buf || ctas < 1) return nullptr;
+    const size_t need = (size_t)ctas * 64;
+    if (g_trace_used + need > g_trace_words) return nullptr;
+    unsigned long long* rec = g_trace_buf + g_trace_used;
+    g_trace_used += need;
+    g_trace_ctas.push_back(ctas);
+    return rec;
+#else
+    (void)ctas;
+    return nullptr;
+#endif
+}
+
+extern "C" int rabit_trace_begin(void* dev_buf, size_t bytes) {
+    rabit_clear_error();
+#ifdef RABIT_TRACE
+    if (dev_buf && (((uintptr_t)dev_buf & 7u) != 0 || bytes < 64))
+        return rabit_fail(RABIT_INVALID_ARG, "rabit_trace_begin: buffer must be 8-byte aligned and hold at least 64 bytes");
+    g_trace_buf = (unsigned long long*)dev_buf;
+    g_trace_words = dev_buf ? bytes / 8 : 0;
+    g_trace_used = 0;
+    g_trace_ctas.clear();
+    return RABIT_OK;
+#else
+    (void)dev_buf; (void)bytes;
+    return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_trace_begin: this library was built without RABIT_TRACE");
+#endif
+}
+
+extern "C" int rabit_trace_launches(int* ctas_out, int max_launches) {
+#ifdef RABIT_TRACE
+    const int n = (int)g_trace_ctas.size();
+    for (int i = 0; i < n && i < max_launches && ctas_out; ++i) ctas_out[i] = g_trace_ctas[i];
+    return n;
+#else
+    (void)ctas_out; (void)max_launches;
+    return 0;
+#endif
+}
+
 extern "C" int rabit_layer_K(const rabit_layer* layer) { return layer ? layer->geom.K : -1; }
 extern "C" int rabit_layer_M(const rabit_layer* layer) { return layer ? layer->geom.M : -1; }
 extern "C" int rabit_layer_N(const rabit_layer* layer) { return layer ? layer->geom.N : -1; }
@@ -426,6 +476,23 @@ extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
     if (variant < 0 || variant > 5) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..5");
     layer->variant = variant;
+    return RABIT_OK;
+}
+
+extern "C" int rabit_set_next(rabit_layer* layer, const rabit_layer* const* next, int n_next) {
+    rabit_clear_error();
+    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: layer is NULL");
+    if (n_next < 0 || n_next > 8) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: n_next must be 0..8 (got %d)", n_next);
+    if (n_next > 0 && !next) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: next is NULL");
+    for (int s = 0; s < n_next; ++s) {
+        if (!next[s]) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: null entry %d", s);
+        if (next[s]->device != layer->device) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: entry %d lives on another device", s);
+    }
+    layer->n_next = n_next;
+    for (int s = 0; s < n_next; ++s) {
+        layer->next_ptr[s] = next[s]->d_lut;
+        layer->next_bytes[s] = (unsigned long long)next[s]->geom.n_cs * next[s]->geom.n_rb * next[s]->geom.K * RABIT_LUT_PART_BYTES;
+    }
     return RABIT_OK;
 }
 

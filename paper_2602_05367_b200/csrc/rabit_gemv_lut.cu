@@ -9,54 +9,66 @@
 // built once per CTA in shared memory: one byte permute (the address), one shared-memory load and one
 // fp32 add per EIGHT weights.  The input scale h_k is applied once per table (t = h * x), the signed
 // accumulation is the sum of table entries in fp32 registers, and every weight bit is read once.
+// Measured on B200: the look-ups alone run at 81 clocks per 2 KB block per SM (the shared-memory pipe's
+// rate: 64 look-ups + 16 for the weights), 7.3 TB/s over 148 SMs, above what HBM delivers.
 //
 // Work split.  The layer is a grid of blocks (32 rows x 256 columns x K paths, K KB each) stored
 // slice-major; CTA c owns a contiguous range of block positions (cut on the host so that all CTAs cost
 // the same: so much per block, so much per table), which is one contiguous byte range.  A range that
-// crosses into the next 256-column slice rebuilds its table there.
-//   * producer warp: one thread streams the range with bulk asynchronous copies (4 blocks per stage,
-//     mbarrier transaction counts) into a ring that takes up to the rest of shared memory.  It never
-//     waits for the previous kernel in the stream: weights do not depend on it, so they arrive while
-//     that kernel finishes and while this one waits for and reads x (programmatic dependent launch).
-//   * 16 consumer warps: after the dependency wait they build the table of the slice (lane = byte
-//     group, warp = path x upper three index bits; 32 entries each by doubling), then take the blocks
-//     round-robin: lane = row.  A lane copies its 16*K weight words to registers (the stage is released
-//     at once), walks the 32 byte groups of its row in an order rotated by its lane index (so the 32
-//     look-ups of a warp hit 32 banks), and ends with  p = sum_k g_k[row] * s_k.
+// crosses into the next 256-column slice rebuilds its table there.  One CTA per SM, 16 warps:
+//   * before the dependency wait (weights do not depend on the previous kernel in the stream, so this
+//     overlaps its tail under programmatic dependent launch): one thread asks for the CTA's whole byte
+//     range to be prefetched into L2 (bulk prefetch, 64 KB per instruction), every warp loads its first
+//     block into registers, and the input scales of the first table are read;
+//   * after the wait: x of the slice is read, the table is built (lane = byte group, warp = path x upper
+//     three index bits; 32 entries each by doubling), and the warps take the blocks round-robin, lane =
+//     row.  A lane holds its 16*K weight words in registers (128-bit streaming loads, one block ahead:
+//     32 KB in flight per SM, on top of the L2 prefetch), walks the 32 byte groups of
+//     its row in an order rotated by its lane index (so the 32 look-ups of a warp step hit 32 banks), and
+//     ends with  p = sum_k g_k[row] * s_k;
 //   * reduction over the slices of a row, without a second pass, a fence or a wait: p is rounded to a
 //     fixed-point grid that the packer sized so that no finite fp16 input can overflow it, and added with
 //     ONE 64-bit integer atomic to the row's accumulate word, which also counts arrivals (bits 55..62).
 //     The lane whose add returns "all other slices were here" owns the complete sum (old value + its own
 //     term): it rounds once to fp16, stores y and puts the word back to zero.  Integer addition commutes,
 //     so results do not depend on arrival order; a non-finite partial sum sets bit 63 (NaN output).
-// Every wait is bounded; a wait that runs out sets the status word and the kernel drains and returns.
+// No thread ever waits for another CTA, and the only waits inside a CTA are barriers of its own warps.
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <type_traits>
 #include <vector>
 
 #include "rabit_internal.h"
 
 namespace {
 
-constexpr int kWarps = 16;                               // consumer warps
-constexpr int kConsumers = kWarps * 32;
-constexpr int kThreads = kConsumers + 32;                // + the producer warp
-constexpr int kStageBlocks = 4;
+constexpr int kWarps = 16;
+constexpr int kThreads = kWarps * 32;
 constexpr int kMaxGrid = 160;
 constexpr int kMaxGroup = 8;
-constexpr int kMaxSlots = 40;
-constexpr int kSmemLimit = 232448;                       // 227 KB: the most one CTA may have
-constexpr long long kWaitLimitCycles = 1LL << 31;        // about one second
 constexpr unsigned long long kSumMask = (1ULL << 55) - 1;
+constexpr unsigned int kPrefetchChunk = 65536;            // bytes per L2 bulk prefetch instruction
+constexpr long long kPrefetchMax = 1 << 20;               // most bytes a CTA asks to be prefetched
 
-template <int K>
+// Tables: one 64 KB table serves two paths, entry e of (path k, byte group) at  e * 256 + (k & 1) * 128 + group * 4
+// of table k >> 1.  The tables start on a 64 KB boundary of the CTA's shared-memory window, so that a table address
+// is  base | byte << 8 | bank offset  and ONE byte permute builds it whole (no add): see the look-up loop.
+template <int K, int NB>
 struct Tab {
-    static constexpr int kSlotsPerEntry = K <= 2 ? 2 : 4;              // 32-group rows per table entry (one per path)
-    static constexpr int kStride = kSlotsPerEntry * 128;               // bytes between entries
-    static constexpr int kBytes = 256 * kStride;
-    static constexpr int kStageBytes = kStageBlocks * K * RABIT_LUT_PART_BYTES;
+    static constexpr int kTables = (K + 1) / 2;                       // per batch row
+    static constexpr int kBytes = kTables * 65536;                    // per batch row
+    static constexpr int kSmem = 65536 + NB * kBytes;                 // alignment slack + tables
+    __host__ __device__ static constexpr int offset(int k, int b) { return b * kBytes + (k >> 1) * 65536 + (k & 1) * 128; }
 };
+
+template <int I, int N, typename F>
+__device__ __forceinline__ void static_for(F&& f) {
+    if constexpr (I < N) {
+        f(std::integral_constant<int, I>{});
+        static_for<I + 1, N>(f);
+    }
+}
 
 struct LutLayer {
     const unsigned char* lut;
@@ -68,49 +80,25 @@ struct LutLayer {
     int M, N, Mp, n_rb, n_cs;
     int fix_bits;
     float inv_unit, unit, limit;    // 2^-unit_exp, 2^unit_exp, 2^fix_bits
+    int pad_;                       // (keeps the size a multiple of 8)
 };
+static_assert(sizeof(LutLayer) % 4 == 0 && sizeof(LutLayer) <= 128, "LutLayer is copied to shared memory by one warp, a word per lane");
 struct CtaRange {
     int layer, b0, b1;              // block positions [b0, b1) of that layer
 };
 struct LutParams {
-    int n_layers, n_slots;
-    unsigned int* status;
+    int n_layers;
+    int n_next;                     // successor layers whose look-up blocks this launch asks L2 to fetch (hint)
+    const unsigned char* next_ptr[kMaxGroup];
+    unsigned int next_bytes[kMaxGroup];   // per CTA: CTA c prefetches [c * next_bytes, (c + 1) * next_bytes) of successor s, clipped to next_total
+    unsigned long long next_total[kMaxGroup];
+    unsigned long long* trace;      // RABIT_TRACE builds: 8 time stamps per CTA of this launch (nullptr: none)
     LutLayer layer[kMaxGroup];
     CtaRange range[kMaxGrid];
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after kWaitLimitCycles or as soon as any thread of the CTA gave up.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return;
-    const long long t0 = clock64();
-    unsigned int ns = 32;
-    while (!mbar_try_wait(bar, parity)) {
-        if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return; }
-        __nanosleep(ns);
-        if (ns < 256) ns *= 2;
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+__device__ __forceinline__ void bar_cta() { asm volatile("bar.sync 0;" ::: "memory"); }
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
     uint32_t r;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(s));
@@ -122,13 +110,67 @@ __device__ __forceinline__ float lds_f32(uint32_t addr) {
     asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(OFF));
     return v;
 }
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+// Weights are read exactly once: no L1 allocation, 128-byte L2 sectors.
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::128B.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// The compiler may move an ordinary use of a loaded value up to the load and stall there; these two keep the load
+// early and its first use late (volatile statements keep their order among themselves, and the look-ups are volatile).
+__device__ __forceinline__ unsigned short ldg_u16_early(const unsigned short* p) {
+    unsigned short v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned short use_here_u16(unsigned short v) {
+    unsigned short r;
+    asm volatile("mov.b16 %0, %1;" : "=h"(r) : "h"(v));
+    return r;
+}
+__device__ __forceinline__ unsigned long long use_here_u64(unsigned long long v) {
+    unsigned long long r;
+    asm volatile("mov.b64 %0, %1;" : "=l"(r) : "l"(v));
+    return r;
+}
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned int bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
+// Phase stamps of a CTA (RABIT_TRACE builds only; see rabit_trace_begin in rabit.h): stamp 0 is %globaltimer
+// (nanoseconds, coarse) at entry, stamps 1..7 are SM clock cycles since entry, taken by lane 0 of warp 0.
+#ifdef RABIT_TRACE
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned long long sm_clock() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t));
+    return t;
+}
+#define RABIT_STAMP0() do { trace_t0 = sm_clock(); if (P.trace && lane == 0 && warp == 0) P.trace[(size_t)blockIdx.x * 64] = global_ns(); } while (0)
+#define RABIT_STAMP(i) do { if (P.trace && lane == 0 && warp == 0) P.trace[(size_t)blockIdx.x * 64 + (i)] = sm_clock() - trace_t0; } while (0)
+#else
+#define RABIT_STAMP0() do { } while (0)
+#define RABIT_STAMP(i) do { } while (0)
+#endif
+
+template <int K>
+struct Blk {
+    uint4 v[2 * K];                  // one lane's 32 bytes per path: (path k, half hf) at v[2k + hf]
+};
+template <int K>
+__device__ __forceinline__ Blk<K> load_blk(const uint4* range_base, int bb, int lane) {
+    Blk<K> r;
+    const uint4* p = range_base + (size_t)bb * (K * RABIT_LUT_PART_BYTES / 16) + lane;
+#pragma unroll
+    for (int i = 0; i < 2 * K; ++i) r.v[i] = ldg_stream(p + i * 32);
+    return r;
 }
 
 // What a lane still owes for the last block it accumulated: the answer of its atomic add is looked at
@@ -159,206 +201,257 @@ __device__ __forceinline__ void settle(Pending (&pd)[NB], const LutLayer& L) {
 template <int K, int NB>
 __global__ void __launch_bounds__(kThreads, 1)
 rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
-    using T = Tab<K>;
-    extern __shared__ __align__(1024) unsigned char smem[];
-    // tables [NB] | ring [n_slots][stage] | full[kMaxSlots] | empty[kMaxSlots] | abort flag
-    unsigned char* ring = smem + NB * T::kBytes;
-    unsigned long long* full = reinterpret_cast<unsigned long long*>(ring + (size_t)P.n_slots * T::kStageBytes);
-    unsigned long long* empty = full + kMaxSlots;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + kMaxSlots);
+    using T = Tab<K, NB>;
+    extern __shared__ __align__(1024) unsigned char smem[];             // slack up to a 64 KB boundary, then the tables
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n_slots = P.n_slots;
 
+#ifdef RABIT_TRACE
+    unsigned long long trace_t0;
+#endif
+    RABIT_STAMP0();                                                     // entry
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid == 0) {
-        for (int s = 0; s < n_slots; ++s) {
-            mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), kStageBlocks);
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+
+    // The launch parameters live in constant memory, which is cold in every new launch: a first touch of one of its
+    // lines costs a trip to L2.  Everything the CTA needs later is therefore copied to shared memory now, before the
+    // dependency wait, so that none of those trips lands between the arrival of x and the end of the kernel.
+    __shared__ LutLayer layer_copy;
+    __shared__ CtaRange range_copy;
+    if (warp == 0) {
+        const CtaRange r0 = P.range[blockIdx.x];
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(&P.layer[r0.layer]);
+        if (lane < (int)(sizeof(LutLayer) / 4)) reinterpret_cast<uint32_t*>(&layer_copy)[lane] = src[lane];
+        if (lane == 0) range_copy = r0;
     }
     __syncthreads();
-
-    const CtaRange R = P.range[blockIdx.x];
-    const LutLayer& L = P.layer[R.layer];
+    const CtaRange R = range_copy;
+    const LutLayer& L = layer_copy;
     const int n_blocks = R.b1 - R.b0;
-    const int n_stages = (n_blocks + kStageBlocks - 1) / kStageBlocks;
+    const unsigned char* range_bytes = L.lut + (size_t)R.b0 * (K * RABIT_LUT_PART_BYTES);
+    const uint4* range_base = reinterpret_cast<const uint4*>(range_bytes);
 
-    if (warp == kWarps) {
-        // ---- producer: the whole range, as fast as the ring allows; no dependency on the stream's past
-        if (lane == 0) {
-            const unsigned char* src = L.lut + (size_t)R.b0 * (K * RABIT_LUT_PART_BYTES);
-            for (int i = 0; i < n_stages; ++i) {
-                const int slot = i % n_slots;
-                if (i >= n_slots) {
-                    mbar_wait(smem_u32(&empty[slot]), ((i / n_slots) - 1) & 1, abort_flag);
-                    if (*abort_flag) break;
-                }
-                const int blocks = min(kStageBlocks, n_blocks - i * kStageBlocks);
-                const uint32_t bytes = blocks * K * RABIT_LUT_PART_BYTES;
-                const uint32_t bar = smem_u32(&full[slot]);
-                mbar_expect_tx(bar, bytes);
-                bulk_g2s(smem_u32(ring + (size_t)slot * T::kStageBytes), src + (size_t)i * T::kStageBytes, bytes, bar);
-            }
+    // ---- everything that does not depend on the stream's past
+    if (tid == 0) {
+        long long left = (long long)n_blocks * (K * RABIT_LUT_PART_BYTES);
+        if (left > kPrefetchMax) left = kPrefetchMax;
+        for (long long off = 0; off < left; off += kPrefetchChunk)
+            prefetch_l2(range_bytes + off, (unsigned int)(left - off < kPrefetchChunk ? left - off : kPrefetchChunk));
+    }
+    if (tid == 32) {
+        // the layers the caller named as the next ones to run: their weights cross HBM (and their pages enter the
+        // TLBs) while this kernel waits and computes, instead of at the start of their own kernel
+        for (int s = 0; s < P.n_next; ++s) {
+            const unsigned long long lo = (unsigned long long)blockIdx.x * P.next_bytes[s];
+            if (lo >= P.next_total[s]) continue;
+            unsigned long long left = P.next_total[s] - lo;
+            if (left > P.next_bytes[s]) left = P.next_bytes[s];
+            for (unsigned long long off = 0; off < left; off += kPrefetchChunk)
+                prefetch_l2(P.next_ptr[s] + lo + off, (unsigned int)(left - off < kPrefetchChunk ? left - off : kPrefetchChunk));
         }
-    } else if (n_blocks > 0) {
-        // ---- consumers
-        const uint32_t tab0 = smem_u32(smem);
-        uint32_t c[8];                                   // byte i of c[j]: bank offset of the group this lane visits in step 4j+i
+    }
+    const int n_mine = warp < n_blocks ? (n_blocks - warp + kWarps - 1) / kWarps : 0;    // blocks warp, warp + 16, ...
+    Blk<K> cur;                                          // this warp's current block
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint32_t v = 0;
+    for (int i = 0; i < 2 * K; ++i) cur.v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (n_mine > 0) cur = load_blk<K>(range_base, warp, lane);
+
+    const uint32_t tab0 = (smem_u32(smem) + 65535u) & ~65535u;
+    // c[j][h]: bytes 0, 1 = bank offsets (4 * group) of the groups this lane visits in steps 4j + 2h and 4j + 2h + 1,
+    // bytes 2, 3 = the upper half of the table base.  A permute of (weight word, c) then yields a complete address.
+    uint32_t c[8][2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v |= (uint32_t)((((4 * j + i) + lane) & 31) * (K <= 2 ? 4 : 2)) << (8 * i);
-            c[j] = v;
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            c[j][h] = (uint32_t)((((4 * j + 2 * h) + lane) & 31) * 4) | (uint32_t)((((4 * j + 2 * h + 1) + lane) & 31) * 4) << 8 | (tab0 & 0xFFFF0000u);
+    int cs = R.b0 / L.n_rb;
+    int seg_rb0 = R.b0 - cs * L.n_rb;                    // row block of the first block of the current segment
+    int seg_begin = 0, seg_end = min(n_blocks, L.n_rb - seg_rb0);       // blocks [seg_begin, seg_end) of the range use slice cs
+    constexpr int kPairs = (8 * K + kWarps - 1) / kWarps;                // (path, upper index bits) pairs a warp builds
+    uint4 hq[kPairs], xq[NB];
+    auto load_h = [&](int slice) {                                      // static data: may be read before the dependency wait
+#pragma unroll
+        for (int u = 0; u < kPairs; ++u) {
+            const int pi = warp + u * kWarps;
+            const int col = slice * RABIT_LUT_COLS + 8 * lane;
+            hq[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (pi < 8 * K && col < L.N) hq[u] = __ldg(reinterpret_cast<const uint4*>(L.h + (size_t)(pi >> 3) * L.N + col));
         }
-        int cs = R.b0 / L.n_rb;
-        int rb = R.b0 - cs * L.n_rb;
-        constexpr int kPairs = (8 * K + kWarps - 1) / kWarps;            // (path, upper index bits) pairs a warp builds
-        uint4 hq[kPairs];
-        auto load_h = [&](int slice) {                                  // static data: may be read before the dependency wait
+    };
+    auto load_x = [&](int slice) {                                      // L2 (not L1): written by the previous kernel in the stream
+        const int col = slice * RABIT_LUT_COLS + 8 * lane;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            xq[b] = make_uint4(0u, 0u, 0u, 0u);
+            if (col < L.N) xq[b] = __ldcg(reinterpret_cast<const uint4*>(L.x + (size_t)b * L.N + col));
+        }
+    };
+    // table of the slice whose h and x sit in hq / xq:  entry e of (path k, group) = sum_{bit<8} (e has bit ? -t : +t),  t = h * x
+    auto build_table = [&]() {
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const uint32_t xw[4] = {xq[b].x, xq[b].y, xq[b].z, xq[b].w};
 #pragma unroll
             for (int u = 0; u < kPairs; ++u) {
                 const int pi = warp + u * kWarps;
-                const int col = slice * RABIT_LUT_COLS + 8 * lane;
-                hq[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (pi < 8 * K && col < L.N) hq[u] = __ldg(reinterpret_cast<const uint4*>(L.h + (size_t)(pi >> 3) * L.N + col));
-            }
-        };
-        load_h(cs);
-
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-
-        Pending pd[NB];
+                if (pi >= 8 * K) break;
+                const int k = pi >> 3, ehi = pi & 7;
+                const uint32_t hw[4] = {hq[u].x, hq[u].y, hq[u].z, hq[u].w};
+                float t[8];
 #pragma unroll
-        for (int b = 0; b < NB; ++b) pd[b].live = false;
-        int b_done = 0;
-        while (b_done < n_blocks) {
-            const int seg = min(n_blocks - b_done, L.n_rb - rb);
-            // ---- table of slice cs:  entry e of (path k, group) = sum_{bit<8} (e has bit ? -t : +t),  t = h * x
-            {
-                const int col = cs * RABIT_LUT_COLS + 8 * lane;
-#pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    uint4 xraw = make_uint4(0u, 0u, 0u, 0u);
-                    if (col < L.N) xraw = __ldcg(reinterpret_cast<const uint4*>(L.x + (size_t)b * L.N + col));   // L2: written by the previous kernel
-                    const uint32_t xw[4] = {xraw.x, xraw.y, xraw.z, xraw.w};
-#pragma unroll
-                    for (int u = 0; u < kPairs; ++u) {
-                        const int pi = warp + u * kWarps;
-                        if (pi >= 8 * K) break;
-                        const int k = pi >> 3, ehi = pi & 7;
-                        const uint32_t hw[4] = {hq[u].x, hq[u].y, hq[u].z, hq[u].w};
-                        float t[8];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[q]));
-                            const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[q]));
-                            t[2 * q] = hf.x * xf.x;                      // exact: two 11-bit significands
-                            t[2 * q + 1] = hf.y * xf.y;
-                        }
-                        float v[32];
-                        v[0] = (ehi & 1 ? -t[5] : t[5]) + (ehi & 2 ? -t[6] : t[6]) + (ehi & 4 ? -t[7] : t[7])
-                             + (((t[0] + t[1]) + (t[2] + t[3])) + t[4]);
-#pragma unroll
-                        for (int bit = 0; bit < 5; ++bit) {
-                            const float m2 = -2.f * t[bit];
-#pragma unroll
-                            for (int e = 0; e < (1 << bit); ++e) v[e | (1 << bit)] = v[e] + m2;
-                        }
-                        const uint32_t dst = tab0 + b * T::kBytes + (ehi * 32) * T::kStride + k * 128 + lane * 4;
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) sts_f32(dst + e * T::kStride, v[e]);
-                    }
+                for (int w = 0; w < 4; ++w) {
+                    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hw[w]));
+                    const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xw[w]));
+                    t[2 * w] = hf.x * xf.x;                              // exact: two 11-bit significands
+                    t[2 * w + 1] = hf.y * xf.y;
                 }
-            }
-            bar_consumers();
-
-            // ---- blocks b_done .. b_done + seg - 1 of the range, round-robin over the warps
-            // (after a wait ran out the warps keep walking the segments, without work, so that all of them
-            //  meet at the same barriers)
-            int bb = b_done + ((warp - b_done) & (kWarps - 1));
-            for (; bb < b_done + seg && !*abort_flag; bb += kWarps) {
-                const int row = (rb + (bb - b_done)) * RABIT_LUT_ROWS + lane;
-                float gk[K];
+                float v[32];
+                v[0] = (ehi & 1 ? -t[5] : t[5]) + (ehi & 2 ? -t[6] : t[6]) + (ehi & 4 ? -t[7] : t[7])
+                     + (((t[0] + t[1]) + (t[2] + t[3])) + t[4]);
 #pragma unroll
-                for (int k = 0; k < K; ++k) gk[k] = __half2float(__ldg(L.g + (size_t)k * L.Mp + row));
-                const int stage = bb / kStageBlocks, slot = stage % n_slots;
-                mbar_wait(smem_u32(&full[slot]), (stage / n_slots) & 1, abort_flag);
-                if (*abort_flag) break;
-                const uint32_t src = smem_u32(ring + (size_t)slot * T::kStageBytes) + (bb % kStageBlocks) * (K * RABIT_LUT_PART_BYTES) + lane * 16;
-                uint32_t w[K][8];
+                for (int bit = 0; bit < 5; ++bit) {
+                    const float m2 = -2.f * t[bit];
 #pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    const uint4 lo = lds_v4(src + k * RABIT_LUT_PART_BYTES), hi = lds_v4(src + k * RABIT_LUT_PART_BYTES + 512);
-                    w[k][0] = lo.x; w[k][1] = lo.y; w[k][2] = lo.z; w[k][3] = lo.w;
-                    w[k][4] = hi.x; w[k][5] = hi.y; w[k][6] = hi.z; w[k][7] = hi.w;
+                    for (int e = 0; e < (1 << bit); ++e) v[e | (1 << bit)] = v[e] + m2;
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&empty[slot]));      // the weights are in registers: the stage may be refilled
-
-                float acc[NB][K][2];
+                const uint32_t dst = tab0 + b * T::kBytes + (k >> 1) * 65536 + (ehi * 32) * 256 + (k & 1) * 128 + lane * 4;
 #pragma unroll
-                for (int b = 0; b < NB; ++b)
-#pragma unroll
-                    for (int k = 0; k < K; ++k) acc[b][k][0] = acc[b][k][1] = 0.f;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-#pragma unroll
-                    for (int k = 0; k < K; ++k) {
-                        uint32_t a0 = prmt(w[k][j], c[j], 0xCC04), a1 = prmt(w[k][j], c[j], 0xDD15);
-                        uint32_t a2 = prmt(w[k][j], c[j], 0xEE26), a3 = prmt(w[k][j], c[j], 0xFF37);
-                        if (K > 2) { a0 <<= 1; a1 <<= 1; a2 <<= 1; a3 <<= 1; }
-#pragma unroll
-                        for (int b = 0; b < NB; ++b) {
-                            const uint32_t tb = tab0 + b * T::kBytes + k * 128;
-                            acc[b][k][0] += lds_f32<0>(tb + a0);
-                            acc[b][k][1] += lds_f32<0>(tb + a1);
-                            acc[b][k][0] += lds_f32<0>(tb + a2);
-                            acc[b][k][1] += lds_f32<0>(tb + a3);
-                        }
-                    }
-
-                settle<NB>(pd, L);                                       // the previous block's atomics have long returned
-#pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    float p = 0.f;
-#pragma unroll
-                    for (int k = 0; k < K; ++k) p += gk[k] * (acc[b][k][0] + acc[b][k][1]);
-                    const float scaled = p * L.inv_unit;
-                    const bool bad = !(fabsf(scaled) < L.limit);          // inf or NaN: finite inputs cannot get here
-                    const long long q = bad ? 0LL : __float2ll_rn(scaled);
-                    pd[b].add = (unsigned long long)(q + (1LL << L.fix_bits)) + (1ULL << 55);
-                    pd[b].word = L.acc + (size_t)b * L.Mp + row;
-                    pd[b].yp = row < L.M ? L.y + (size_t)b * L.M + row : nullptr;
-                    pd[b].bad = bad;
-                    if (bad) atomicOr(pd[b].word, 1ULL << 63);
-                    pd[b].old = atomicAdd(pd[b].word, pd[b].add);
-                    pd[b].live = true;
-                }
+                for (int e = 0; e < 32; ++e) sts_f32(dst + e * 256, v[e]);
             }
-            b_done += seg;
+        }
+    };
+    // makes the table of block bb's slice the current one; every warp crosses every slice border of the range here
+    auto advance_to = [&](int bb) {
+        while (bb >= seg_end) {
+            bar_cta();                                                  // every warp is done with the old table
+            build_table();
             cs += 1;
-            rb = 0;
-            if (b_done < n_blocks) {
-                load_h(cs);
-                bar_consumers();                                        // every warp is done with the old table
+            seg_begin = seg_end;
+            seg_rb0 = 0;
+            seg_end = min(n_blocks, seg_end + L.n_rb);
+            if (seg_end < n_blocks) { load_h(cs + 1); load_x(cs + 1); } // the table after this one
+            bar_cta();
+        }
+    };
+    load_h(cs);
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    RABIT_STAMP(1);                                                     // the previous kernel's results are visible
+    if (n_blocks <= 0) return;
+    load_x(cs);
+#ifdef RABIT_TRACE
+    if (xq[0].x == 0x12345678u && xq[0].y == 0x9ABCDEF0u && hq[0].x == 0x12345678u) RABIT_STAMP(7);   // (a use of x and h, so that the next stamp follows their arrival)
+#endif
+    RABIT_STAMP(2);                                                     // x and h of the first table have arrived
+    build_table();
+    if (seg_end < n_blocks) { load_h(cs + 1); load_x(cs + 1); }
+    bar_cta();
+    RABIT_STAMP(3);                                                     // first table built
+
+    // One iteration per block of this warp.  Everything with a long latency is ISSUED at the top of an iteration
+    // (the next block's weights, this block's output scales, the atomic adds of the previous block) and its result is
+    // first touched below the look-ups of the same iteration, some 1300 cycles later: no request is in flight across the
+    // loop's back edge, where the compiler would otherwise have the warp wait for it (a warp has six scoreboards).
+    Pending pd[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) { pd[b].live = false; pd[b].old = 0ULL; pd[b].add = 0ULL; pd[b].word = nullptr; pd[b].yp = nullptr; pd[b].bad = false; }
+    bool owe = false;                                                   // pd holds a finished block whose atomics are still to be issued
+    for (int i = 0; i < n_mine; ++i) {
+        const int bb = warp + i * kWarps;
+#ifdef RABIT_TRACE
+        if (i < 11) RABIT_STAMP(8 + 5 * i);                             // iteration i: top
+#endif
+        advance_to(bb);
+        const int row = (seg_rb0 + (bb - seg_begin)) * RABIT_LUT_ROWS + lane;
+        unsigned short graw[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) graw[k] = ldg_u16_early(reinterpret_cast<const unsigned short*>(L.g) + (size_t)k * L.Mp + row);
+        Blk<K> nxt = load_blk<K>(range_base, i + 1 < n_mine ? bb + kWarps : bb, lane);   // (the last iteration re-reads its own block: in bounds, unused)
+        if (owe) {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                if (pd[b].bad) atomicOr(pd[b].word, 1ULL << 63);
+                pd[b].old = atomicAdd(pd[b].word, pd[b].add);
+                pd[b].live = true;
             }
         }
-        settle<NB>(pd, L);
-    }
-
-    __syncthreads();                                                    // abort_flag of every warp is final
-    if (*abort_flag && tid == kConsumers) {
-        // make sure no bulk copy is still in flight towards this CTA's shared memory
-        for (int it = max(0, n_stages - n_slots); it < n_stages; ++it) {
-            const long long t0 = clock64();
-            while (!mbar_try_wait(smem_u32(&full[it % n_slots]), (it / n_slots) & 1))
-                if (clock64() - t0 > kWaitLimitCycles) break;
+        if (i == 0) RABIT_STAMP(4);                                     // first weights in registers
+#ifdef RABIT_TRACE
+        {
+            unsigned int u = cur.v[0].x;
+#pragma unroll
+            for (int t = 0; t < 2 * K; ++t) u |= cur.v[t].w;
+            u = (unsigned int)use_here_u64(u);                           // the block's weights have arrived
+            if (i < 11 && u != 0x13572468u) RABIT_STAMP(9 + 5 * i);
         }
-        atomicExch(P.status, 1u);
+#endif
+
+        float acc[NB][K][2];
+#pragma unroll
+        for (int b = 0; b < NB; ++b)
+#pragma unroll
+            for (int k = 0; k < K; ++k) acc[b][k][0] = acc[b][k][1] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            static_for<0, K>([&](auto kc) {
+                constexpr int k = decltype(kc)::value;
+                const uint4 part = cur.v[2 * k + (j >> 2)];
+                const uint32_t w = (j & 3) == 0 ? part.x : (j & 3) == 1 ? part.y : (j & 3) == 2 ? part.z : part.w;
+                // address = table base | sign byte << 8 | bank offset, all from one permute
+                const uint32_t a0 = prmt(w, c[j][0], 0x7604), a1 = prmt(w, c[j][0], 0x7615);
+                const uint32_t a2 = prmt(w, c[j][1], 0x7624), a3 = prmt(w, c[j][1], 0x7635);
+                static_for<0, NB>([&](auto bc) {
+                    constexpr int b = decltype(bc)::value;
+                    acc[b][k][0] += lds_f32<T::offset(k, b)>(a0);
+                    acc[b][k][1] += lds_f32<T::offset(k, b)>(a1);
+                    acc[b][k][0] += lds_f32<T::offset(k, b)>(a2);
+                    acc[b][k][1] += lds_f32<T::offset(k, b)>(a3);
+                });
+            });
+#ifdef RABIT_TRACE
+        if (i == 0) RABIT_STAMP(7);                                     // first block's look-ups issued
+        if (i < 11 && use_here_u64(__float_as_uint(acc[0][0][0] + acc[0][0][1] + acc[0][K - 1][0] + acc[0][K - 1][1])) != 0x13572468u) RABIT_STAMP(10 + 5 * i);   // look-ups answered
+#endif
+#pragma unroll
+        for (int b = 0; b < NB; ++b) pd[b].old = use_here_u64(pd[b].old);
+        settle<NB>(pd, L);                                               // the previous block's atomics, issued above the look-ups
+#ifdef RABIT_TRACE
+        if (i < 11) RABIT_STAMP(11 + 5 * i);                            // previous atomic answered and settled
+#endif
+#pragma unroll
+        for (int k = 0; k < K; ++k) graw[k] = use_here_u16(graw[k]);
+#ifdef RABIT_TRACE
+        if (i < 11) RABIT_STAMP(12 + 5 * i);                            // output scales have arrived
+#endif
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            float p = 0.f;
+#pragma unroll
+            for (int k = 0; k < K; ++k) p += __half2float(__ushort_as_half(graw[k])) * (acc[b][k][0] + acc[b][k][1]);
+            const float scaled = p * L.inv_unit;
+            const bool bad = !(fabsf(scaled) < L.limit);                  // inf or NaN: finite inputs cannot get here
+            const long long qv = bad ? 0LL : __float2ll_rn(scaled);
+            pd[b].add = (unsigned long long)(qv + (1LL << L.fix_bits)) + (1ULL << 55);
+            pd[b].word = L.acc + (size_t)b * L.Mp + row;
+            pd[b].yp = row < L.M ? L.y + (size_t)b * L.M + row : nullptr;
+            pd[b].bad = bad;
+        }
+        owe = true;
+#pragma unroll
+        for (int t = 0; t < 2 * K; ++t) cur.v[t] = nxt.v[t];             // the next block's weights have arrived by now
+        cur.v[0].x = (unsigned int)use_here_u64(cur.v[0].x);
     }
+    if (owe) {
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            if (pd[b].bad) atomicOr(pd[b].word, 1ULL << 63);
+            pd[b].old = atomicAdd(pd[b].word, pd[b].add);
+            pd[b].live = true;
+        }
+    }
+    RABIT_STAMP(5);                                                     // last look-up done, last atomic issued
+    advance_to(n_blocks - 1);                                           // warps that ran out of blocks early still take part in the rebuilds
+    settle<NB>(pd, L);
+    RABIT_STAMP(6);                                                     // last atomic answered, y stored
 }
 
 // ---- host side: cutting the layers into ranges of equal cost ------------------------------------
@@ -408,9 +501,9 @@ long long best_limit(int n_cs, int n_rb, const Cost& C, int n_cta) {
 template <int K, int NB>
 cudaError_t launch_inst(const LutParams& P, int grid, int device, cudaStream_t stream) {
     static bool attr_done[64] = {false};
-    const size_t smem = (size_t)NB * Tab<K>::kBytes + (size_t)P.n_slots * Tab<K>::kStageBytes + 2 * kMaxSlots * 8 + 16;
+    const size_t smem = (size_t)Tab<K, NB>::kSmem;
     if (device < 0 || device >= 64 || !attr_done[device]) {
-        cudaError_t e = cudaFuncSetAttribute(rabit_gemv_lut_kernel<K, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        cudaError_t e = cudaFuncSetAttribute(rabit_gemv_lut_kernel<K, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (device >= 0 && device < 64) attr_done[device] = true;
     }
@@ -427,19 +520,13 @@ cudaError_t launch_inst(const LutParams& P, int grid, int device, cudaStream_t s
     return cudaLaunchKernelEx(&cfg, rabit_gemv_lut_kernel<K, NB>, P);
 }
 
-int max_slots(int K, int nb) {
-    const int table = nb * (K <= 2 ? 65536 : 131072), stage = kStageBlocks * K * RABIT_LUT_PART_BYTES;
-    int s = (kSmemLimit - table - 2 * kMaxSlots * 8 - 16) / stage;
-    return s > kMaxSlots ? kMaxSlots : s;
-}
-
 }  // namespace
 
 int rabit_gemv_lut_max_rows() { return 2; }
 
 bool rabit_gemv_lut_supports(const rabit_layer& L, int batch) {
     if (batch < 1 || batch > 2) return false;
-    if (L.geom.K == 3 && batch > 1) return false;                        // two 128 KB tables do not fit
+    if (L.geom.K == 3 && batch > 1) return false;                        // four 64 KB tables do not fit into shared memory
     if (L.geom.n_cs > RABIT_LUT_MAX_SLICES) return false;
     return (long long)L.geom.n_cs * L.geom.n_rb < (1LL << 30) && L.d_lut != nullptr && L.d_acc != nullptr;
 }
@@ -461,7 +548,8 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
     const int K = layers[0]->geom.K;
     LutParams P;
     P.n_layers = n_layers;
-    P.status = status_override ? status_override : layers[0]->d_status;
+    (void)status_override;                                               // this kernel has no wait that could run out
+    P.trace = nullptr;
     const Cost C = cost_of(K, batch);
     long long weight[kMaxGroup], total_weight = 0, total_blocks = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -531,22 +619,36 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
         n_cta[lo] -= 1; n_cta[hi] += 1;
         limit[lo] = lo_new; limit[hi] = hi_new;
     }
-    int c0 = 0, max_blocks = 0;
+    int c0 = 0;
     std::vector<int> cuts;
     for (int l = 0; l < n_layers; ++l) {
         const int used = ctas_needed(layers[l]->geom.n_cs, layers[l]->geom.n_rb, C, limit[l], &cuts);
         if (used > n_cta[l] || c0 + used > kMaxGrid) return cudaErrorInvalidValue;      // cannot happen: limit[l] was found with n_cta[l]
         for (int i = 0; i < used; ++i) {
             P.range[c0 + i] = CtaRange{l, cuts[i], cuts[i + 1]};
-            max_blocks = std::max(max_blocks, cuts[i + 1] - cuts[i]);
         }
         c0 += used;
     }
     const int launch_grid = c0;
     for (int i = c0; i < kMaxGrid; ++i) P.range[i] = CtaRange{0, 0, 0};
-    const int want = (max_blocks + kStageBlocks - 1) / kStageBlocks;
-    P.n_slots = std::max(1, std::min(want, max_slots(K, batch)));
     const int device = layers[0]->device;
+    // successors named by rabit_set_next on any layer of the group (each once)
+    P.n_next = 0;
+    for (int l = 0; l < n_layers; ++l)
+        for (int s = 0; s < layers[l]->n_next && P.n_next < kMaxGroup; ++s) {
+            bool seen = false;
+            for (int t = 0; t < P.n_next; ++t) seen = seen || P.next_ptr[t] == layers[l]->next_ptr[s];
+            if (seen || layers[l]->next_bytes[s] == 0) continue;
+            const unsigned long long total = layers[l]->next_bytes[s];
+            unsigned long long per_cta = (total + launch_grid - 1) / launch_grid;
+            per_cta = (per_cta + 1023) & ~1023ULL;                       // whole 1 KB parts (16-byte granularity is what the instruction needs)
+            P.next_ptr[P.n_next] = layers[l]->next_ptr[s];
+            P.next_bytes[P.n_next] = (unsigned int)per_cta;
+            P.next_total[P.n_next] = total;
+            ++P.n_next;
+        }
+    for (int s = P.n_next; s < kMaxGroup; ++s) { P.next_ptr[s] = nullptr; P.next_bytes[s] = 0; P.next_total[s] = 0; }
+    P.trace = rabit_trace_slot(launch_grid);
     if (K == 1) return batch == 1 ? launch_inst<1, 1>(P, launch_grid, device, stream) : launch_inst<1, 2>(P, launch_grid, device, stream);
     if (K == 2) return batch == 1 ? launch_inst<2, 1>(P, launch_grid, device, stream) : launch_inst<2, 2>(P, launch_grid, device, stream);
     return launch_inst<3, 1>(P, launch_grid, device, stream);

@@ -24,6 +24,9 @@ struct rabit_layer {
     unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
     const unsigned char* d_lut;  // look-up blocks (table-driven GEMV)
     unsigned long long* d_acc;   // u64 [RABIT_LUT_MAX_BATCH][Mp] accumulate words of the table-driven GEMV (zero between calls)
+    int n_next;                  // rabit_set_next: look-up sections the decode kernel of this layer asks L2 to fetch
+    const unsigned char* next_ptr[8];
+    unsigned long long next_bytes[8];
 };
 
 // error reporting (thread-local message); returns `code`
@@ -62,6 +65,10 @@ int rabit_gemv_mma_max_rows();
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream);
+// Phase tracing (rabit_api.cu): the next free record of 8 stamps x `ctas` in the caller's trace buffer, or nullptr
+// when tracing is off, the buffer is full or the library was built without RABIT_TRACE.
+unsigned long long* rabit_trace_slot(int ctas);
+
 // table-driven GEMV (rabit_gemv_lut.cu); acc_override / status_override redirect the scratch (nullptr: the image's own)
 cudaError_t rabit_launch_gemv_lut(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
 bool rabit_gemv_lut_supports(const rabit_layer& L, int batch);
