@@ -29,11 +29,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of the four launches of one grouped step, from the ncu capture summarised in
-# profiles/gemv_mma_llama2_7b_decoder_layer.md (12.759 + 4.296 + 22.771 + 11.417 MB); valid for the
-# default grouped batch-1 workload only.
-NCU_DRAM_BYTES_PER_GROUPED_STEP = 51_272_192
-
 METRIC = "batch-1 residual-binary GEMV us/layer"
 UNIT = "us/layer"
 WORKLOAD = "llama2-7b decoder layer: 7 residual-binary projections, K=2, batch 1, back to back"
@@ -169,6 +164,85 @@ def run_step(rabit, shapes, layer_row, xs, ys, token: int, grouped: bool = True)
 
 
 # ---------------------------------------------------------------------------------------
+# timing helpers
+# ---------------------------------------------------------------------------------------
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops", 1590.0)),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 1400.0)), "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def recorded_traffic(key: str):
+    """DRAM bytes per step from the ncu capture recorded in profiles/gemv_lut_traffic.json, or None when no capture of
+    this workload is on record there (the file names the command and the kernel source it was taken with)."""
+    path = os.path.join(ROOT, "profiles", "gemv_lut_traffic.json")
+    try:
+        rec = json.load(open(path))
+    except (OSError, ValueError):
+        return None
+    entry = rec.get(key)
+    return None if entry is None else entry.get("dram_bytes_per_step")
+
+
+def time_replays(stream, graphs, repeats: int, warm: int = 1):
+    """Milliseconds of `repeats` timed passes over the list of CUDA graphs (each pass replays every graph once, in
+    order), CUDA events on the launching stream; `warm` untimed passes first."""
+    import torch
+    out = []
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            for g in graphs:
+                g.replay()
+    stream.synchronize()
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for g in graphs:
+                g.replay()
+            e1.record(stream)
+        stream.synchronize()
+        out.append(e0.elapsed_time(e1))
+    return out
+
+
+def capture_graph(stream, fn):
+    import torch
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        fn()
+    return g
+
+
+def measure_stream_read(device, stream) -> float:
+    """Read-only streaming bandwidth in GB/s: 128-bit loads over 2 GiB, best of 5 (the library's own probe kernel)."""
+    import ctypes
+    import torch
+    from paper_2602_05367_b200 import binding
+    lib = binding.raw_lib()
+    n = 2 << 30
+    buf = torch.empty(n, dtype=torch.uint8, device=device)
+    buf.fill_(3)
+    best = None
+    for _ in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            rc = lib.rabit_selftest_stream_read(ctypes.c_void_p(buf.data_ptr()), n, None, ctypes.c_void_p(stream.cuda_stream))
+            e1.record(stream)
+        stream.synchronize()
+        assert rc == 0
+        ms = e0.elapsed_time(e1)
+        best = ms if best is None or ms < best else best
+    del buf
+    torch.cuda.empty_cache()
+    return n / (best * 1e-3) / 1e9
+
+
+# ---------------------------------------------------------------------------------------
 # the library arm
 # ---------------------------------------------------------------------------------------
 def bench_rabit(args) -> dict:
@@ -193,78 +267,78 @@ def bench_rabit(args) -> dict:
             dist.barrier()
         torch.cuda.synchronize()
 
-    copies, batch, tokens = args.copies, args.batch, 16
-    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens, hints=not args.no_hints)
+    copies, batch, tokens = args.copies, args.batch, 4
+    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens, hints=args.hints)
     step_bytes = sum(layer_bytes(sh.M, sh.N, batch) for sh in shapes)
     n_proj = len(shapes)
     stream = torch.cuda.Stream(device)
-
-    # one CUDA graph per decoder-layer copy, and one that walks all copies once
-    def capture(copy_ids):
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=stream):
-            for c in copy_ids:
-                run_step(rabit, shapes, layers[c], xs, ys, c % tokens, grouped)
-        return g
-
     grouped = not args.no_group
     launches_per_step = len(GROUPS) if grouped else n_proj
+    peaks = load_peaks()
+
+    def steps_fn(first: int, count: int):
+        """Steps first .. first+count-1; step s runs decoder-layer copy s % copies on the current token's activations (a
+        token's hidden state is re-read by every layer of the stack, so it is warm in L2; the weights are not)."""
+        def fn():
+            for s in range(first, first + count):
+                run_step(rabit, shapes, layers[s % copies], xs, ys, 0, grouped)
+        return fn
+
     with torch.cuda.stream(stream):
-        for c in range(copies):                      # also the first-call set-up of every kernel variant
-            run_step(rabit, shapes, layers[c], xs, ys, c % tokens, grouped)
+        steps_fn(0, copies)()                        # first-call set-up of every kernel variant, outside any capture
     stream.synchronize()
-    use_graph = not args.no_graph
-    if use_graph:
-        cycle_graph = capture(list(range(copies)))
-        step_graphs = [capture([c]) for c in range(copies)]
 
-    def run_steps(first: int, count: int):
-        """Steps first .. first+count-1; step s uses decoder-layer copy s % copies."""
-        s, end = first, first + count
-        with torch.cuda.stream(stream):
-            while s < end:
-                if not use_graph:
-                    run_step(rabit, shapes, layers[s % copies], xs, ys, (s % copies) % tokens, grouped)
-                    s += 1
-                elif s % copies == 0 and end - s >= copies:
-                    cycle_graph.replay(); s += copies
-                else:
-                    step_graphs[s % copies].replay(); s += 1
+    # The timed region is K steps as whole CUDA graphs, whatever K is: full cycles over the copies replay one graph of
+    # `copies` steps, the remainder is one graph of its own, so 20 steps and 32000 steps time the same launch pattern.
+    def graphs_for(first: int, count: int):
+        out = []
+        full, rem = divmod(count, copies)
+        if full:
+            cyc = capture_graph(stream, steps_fn(first, copies))
+            out += [cyc] * full
+        if rem:
+            out.append(capture_graph(stream, steps_fn(first + full * copies, rem)))
+        return out
 
+    warm_graphs = graphs_for(0, args.warmup)
+    timed_graphs = graphs_for(args.warmup, args.steps)
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    run_steps(0, args.warmup)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    time_replays(stream, warm_graphs, repeats=0, warm=1)
     barrier()
     t_wall0 = time.time()
-    with torch.cuda.stream(stream):
-        ev0.record(stream)
-    run_steps(args.warmup, args.steps)
-    with torch.cuda.stream(stream):
-        ev1.record(stream)
+    times = time_replays(stream, timed_graphs, repeats=args.repeats, warm=0)
     barrier()
     t_wall1 = time.time()
-    ms = max_over_ranks(ev0.elapsed_time(ev1), dist, device)
+    times = [max_over_ranks(t, dist, device) for t in times]
+    ms = float(np.median(times))
     clocks = sampler.summary(t_wall0, t_wall1) if sampler else None
     if sampler and clocks["samples"] < 3:
         # the timed region was shorter than the sampling period: repeat the same work, untimed,
         # for about a second under the sampler and report the clocks seen there
         reps = max(1, int(1.0 / max(ms * 1e-3, 1e-4)))
         t0 = time.time()
-        for _ in range(reps):
-            run_steps(args.warmup, args.steps)
-        torch.cuda.synchronize()
+        time_replays(stream, timed_graphs, repeats=0, warm=reps)
         clocks = sampler.summary(t0, time.time())
         clocks["note"] = "sampled over an untimed repeat of the timed region (region shorter than the sampler period)"
     if sampler:
         sampler.stop()
 
     ms_per_step = ms / args.steps
-    us_per_layer = ms_per_step * 1e3 / n_proj
     gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    gbs_best = step_bytes / (min(times) / args.steps * 1e-3) / 1e9
+
+    # ---- warm-L2 figure (labelled; the paper's own latencies are warm-cache): one decoder layer, 51 MB, replayed in place
+    warm_l2 = None
+    if rank == 0 and world == 1 and not args.no_extras:
+        g1 = capture_graph(stream, steps_fn(0, 1))
+        t = time_replays(stream, [g1] * 200, repeats=5, warm=2)
+        warm_l2 = {"us_per_layer": float(np.median(t)) / 200 * 1e3 / n_proj, "gbs_equivalent": step_bytes / (float(np.median(t)) / 200 * 1e-3) / 1e9,
+                   "note": "the same step replayed on ONE decoder layer: its 51 MB stay in the 126 MB L2, no HBM traffic"}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     e2e = None
     if rank == 0 or dist is not None:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         pin_x = {n: torch.from_numpy(a).pin_memory() for n, a in xs_host.items()}
         pin_y = [torch.empty((batch, sh.M), dtype=torch.float16).pin_memory() for sh in shapes]
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -287,7 +361,6 @@ def bench_rabit(args) -> dict:
         for s in range(min(3 * copies, 100)):
             e2e_step(s)
         barrier()
-        t0 = time.perf_counter()
         with torch.cuda.stream(stream):
             ev0.record(stream)
         for s in range(e2e_steps):
@@ -302,38 +375,47 @@ def bench_rabit(args) -> dict:
                "steps": e2e_steps, "note": ("rabit_linear_group_host (prepared calls) per group of projections (a shared input is copied once)" if grouped else
                         "rabit_linear_host per projection") + ": pinned host x -> device stage by copy, kernel, y stored by the kernel straight into pinned (mapped) host memory, host synchronises after every step"}
 
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    else:
-        peak, peak_src = 6650.0, "fallback"
+    read_peak = measure_stream_read(device, stream) if (rank == 0 and not args.no_extras) else None
+    peak = peaks["hbm_gbs"]
+    traffic_step = recorded_traffic("decoder7b_grouped_batch1") if (grouped and batch == 1) else None
     result = {
         "metric": METRIC, "value": whole_job_us_per_layer(ms_per_step, n_proj, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int8 tensor-core products of exact fixed-point activations, int32/fp32 accumulate, fp16 in/out",
+        "vs_baseline": None, "dtype": "f32 (table look-up sums in fp32 registers, 64-bit fixed-point reduction across CTAs, fp16 in/out)",
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "copies": copies, "batch": batch, "K": K_PATHS,
                    "packed_bytes_total": int(step_bytes * copies),
-                   "l2": "inputs larger than L2: rotation over %d distinct decoder layers (%.0f MB)" % (copies, step_bytes * copies / 1e6),
-                   "launch": "CUDA graph replay" if use_graph else "stream launches",
+                   "l2": "inputs larger than L2: rotation over %d distinct decoder layers (%.0f MB of weights); the activations of the "
+                         "current token are re-read by every layer and stay warm, as in a decoder" % (copies, step_bytes * copies / 1e6),
+                   "launch": "CUDA graph replay: the timed region is whole graphs (one graph per cycle over the copies, one for the remainder)",
                    "launches_per_step": launches_per_step,
+                   "next_layer_prefetch_hints": bool(args.hints),
                    "grouping": "q|k|v and gate|up (projections that share their input) each go through one rabit_linear_group launch; "
                                "o and down through rabit_linear" if grouped else "one rabit_linear launch per projection",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "repeats": {"n": len(times), "ms_median": ms, "ms_min": min(times), "ms_max": max(times),
+                    "us_per_layer_median": ms_per_step * 1e3 / n_proj, "us_per_layer_min": min(times) / args.steps * 1e3 / n_proj},
         "achieved_hbm_gbs": gbs * world,
-        "tokens_per_s_32_layer_stack": world * 1.0 / (32 * ms_per_step * 1e-3),
-        "gpu_launches": args.steps * launches_per_step,
+        "tokens_per_s_32_layer_stack_extrapolated": world * 1.0 / (32 * ms_per_step * 1e-3),
+        "gpu_launches": args.steps * launches_per_step * max(1, len(times)),
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": (NCU_DRAM_BYTES_PER_GROUPED_STEP / launches_per_step) if (grouped and batch == 1) else None,
+                     "traffic": (traffic_step / launches_per_step) if traffic_step else None,
                      "algorithmic_bytes_per_launch": step_bytes / launches_per_step,
-                     "peak_source": peak_src,
-                     "note": "per launch of rabit_gemv_mma_kernel, averaged over the launches of a step: algorithmic bytes of the "
+                     "peak_source": peaks["source"] + " hbm_gbs (copy bandwidth, read+write bytes)",
+                     "frac_best_repeat": gbs_best / peak,
+                     "other_denominators": {"nominal_8000_gbs": gbs / 8000.0,
+                                            "read_only_stream_gbs": read_peak, "frac_of_read_only_stream": (gbs / read_peak) if read_peak else None},
+                     "note": "per launch of rabit_gemv_lut_kernel, averaged over the launches of a step: algorithmic bytes of the "
                              "step / device time of the step (launch gaps included); traffic = ncu dram bytes of the same launches"},
     }
+    if warm_l2:
+        result["warm_l2"] = warm_l2
+    if rank == 0 and world == 1 and not args.no_extras:
+        result["extras"] = bench_extras(args, rabit, device, stream, shapes, layers, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = cpu_baseline(sample_projections=n_proj)
+        result["cpu_baseline"] = cpu_baseline(sample_projections=n_proj, variants=True)
     for row in layers:
         for L in row:
             L.free()
@@ -342,10 +424,126 @@ def bench_rabit(args) -> dict:
     return result if rank == 0 else None
 
 
+def bench_extras(args, rabit, device, stream, shapes, layers, peaks) -> dict:
+    """Compact measurements of the other benchmark configurations, each with its own roofline fraction (same protocol:
+    cold weights by rotation over distinct copies, graph replay, CUDA events, median of 5)."""
+    import torch
+    from synth import make_layer, make_x
+    out = {}
+    hbm = peaks["hbm_gbs"]
+
+    def timed_case(lys, x, y, launches_note=None):
+        def fn():
+            for L in lys:
+                rabit.rabit_linear(L, x, y)
+        with torch.cuda.stream(stream):
+            fn()
+        stream.synchronize()
+        g = capture_graph(stream, fn)
+        reps = max(1, int(2e-3 / (len(lys) * 20e-6)))
+        t = time_replays(stream, [g] * reps, repeats=5, warm=1)
+        return float(np.median(t)) * 1e3 / (reps * len(lys))
+
+    def make_copies(M, N, K, n, cfg):
+        res = []
+        for c in range(n):
+            L = make_layer(M, N, K, key=(cfg, c, M, N, K))
+            res.append(rabit.rabit_pack(L.planes, L.g, L.h, device=device))
+        return res
+
+    def n_copies(M, N, K):
+        return max(2, min(32, int(4 * 126e6 / layer_bytes(M, N, 1, K)) + 1))
+
+    def hbm_case(M, N, K, batch, us):
+        nb = layer_bytes(M, N, batch, K)
+        return {"M": M, "N": N, "K": K, "batch": batch, "us_per_layer": us, "gbs": nb / us / 1e3, "frac": nb / us / 1e3 / hbm}
+
+    # config 0: the 4096 x 4096 layer alone (the q projections of the rotating decoder layers)
+    x4096 = torch.from_numpy(make_x(1, 4096, key=(0, 0))).to(device)
+    y = torch.zeros((1, 4096), dtype=torch.float16, device=device)
+    us = timed_case([row[0] for row in layers], x4096, y)
+    out["config0_4096x4096_batch1"] = hbm_case(4096, 4096, K_PATHS, 1, us)
+
+    # config 2 as stated: the whole stack (copies x 7 projections), 256 sequential tokens, one token = one CUDA graph
+    if len(layers) >= 32:
+        n_tok = 256
+        xs_all = {n: torch.from_numpy(np.stack([make_x(1, n, key=(2, 10_000 + t))[0] for t in range(n_tok)])).to(device) for n in (4096, 11008)}
+        x_cur = {n: torch.zeros((1, n), dtype=torch.float16, device=device) for n in xs_all}
+        idx = torch.zeros(1, dtype=torch.int64, device=device)
+        ys2 = [torch.zeros((1, sh.M), dtype=torch.float16, device=device) for sh in shapes]
+
+        def token_fn():
+            for n in xs_all:                                   # the token's activations: device-side index, advanced inside the graph
+                torch.index_select(xs_all[n], 0, idx, out=x_cur[n])
+            idx.add_(1).remainder_(n_tok)
+            for row in layers:
+                for grp in GROUPS:
+                    if len(grp) == 1:
+                        rabit.rabit_linear(row[grp[0]], x_cur[shapes[grp[0]].N], ys2[grp[0]])
+                    else:
+                        rabit.rabit_linear_group([row[p] for p in grp], [x_cur[shapes[p].N] for p in grp], [ys2[p] for p in grp])
+        with torch.cuda.stream(stream):
+            token_fn()
+        stream.synchronize()
+        idx.zero_()
+        g = capture_graph(stream, token_fn)
+        t = time_replays(stream, [g] * n_tok, repeats=3, warm=0)
+        sec = float(np.median(t)) * 1e-3
+        stack_bytes = len(layers) * sum(layer_bytes(sh.M, sh.N, 1) for sh in shapes)
+        out["config2_stack_256_tokens"] = {"layers": len(layers) * len(shapes), "tokens": n_tok, "tokens_per_s": n_tok / sec,
+                                            "ms_per_token": sec / n_tok * 1e3, "gbs": stack_bytes * n_tok / sec / 1e9,
+                                            "frac": stack_bytes * n_tok / sec / 1e9 / hbm,
+                                            "note": "one token = one CUDA graph of %d launches (plus three tiny launches that select the token's "
+                                                    "activations by a device-side index); tokens/s = 256 / elapsed" % (len(layers) * len(GROUPS))}
+
+    # config 3 / 4 samples at batch 1, batch 16 on the 8B shapes, the batch-512 GEMM, and K = 1 / 3 at 7B shapes
+    extra_hbm = []
+    for (M, N) in [(14336, 4096), (28672, 8192)]:
+        lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 4)
+        x = torch.from_numpy(make_x(1, N, key=(4, 1, N))).to(device)
+        y = torch.zeros((1, M), dtype=torch.float16, device=device)
+        extra_hbm.append(hbm_case(M, N, K_PATHS, 1, timed_case(lys, x, y)))
+        if (M, N) == (28672, 8192):
+            xb = torch.from_numpy(make_x(512, N, key=(4, 512, N))).to(device)
+            yb = torch.zeros((512, M), dtype=torch.float16, device=device)
+            usb = timed_case(lys, xb, yb)
+            tf = 2.0 * 512 * M * N * K_PATHS / usb / 1e6
+            out["gemm_28672x8192_batch512"] = {"us_per_layer": usb, "tflops": tf, "bound": "tensor", "peak": peaks["bf16_tflops_sustained"],
+                                               "frac": tf / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"] + " bf16_tflops_sustained"}
+        for L in lys:
+            L.free()
+        del lys
+    out["batch1_large_layers"] = extra_hbm
+    b16 = []
+    for (M, N) in [(4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336)]:
+        lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 3)
+        for batch in (1, 16):
+            x = torch.from_numpy(make_x(batch, N, key=(3, batch, N))).to(device)
+            y = torch.zeros((batch, M), dtype=torch.float16, device=device)
+            b16.append(hbm_case(M, N, K_PATHS, batch, timed_case(lys, x, y)))
+        for L in lys:
+            L.free()
+        del lys
+    out["llama3_8b_shapes_batch_1_and_16"] = b16
+    kk = []
+    for K in (1, 3):
+        for (M, N) in [(4096, 4096), (11008, 4096)]:
+            lys = make_copies(M, N, K, n_copies(M, N, K), 5)
+            x = torch.from_numpy(make_x(1, N, key=(5, 1, N))).to(device)
+            y = torch.zeros((1, M), dtype=torch.float16, device=device)
+            kk.append(hbm_case(M, N, K, 1, timed_case(lys, x, y)))
+            for L in lys:
+                L.free()
+            del lys
+    out["paths_1_and_3_batch1"] = kk
+    torch.cuda.empty_cache()
+    return out
+
+
 # ---------------------------------------------------------------------------------------
 # the oracle, timed as it stands on the host cores
 # ---------------------------------------------------------------------------------------
-def cpu_baseline(sample_projections: int = 7, repeats: int = 1) -> dict:
+def cpu_baseline(sample_projections: int = 7, repeats: int = 1, variants: bool = False) -> dict:
     from oracle import rabit_oracle as orc
     from synth import llama2_7b_layer_shapes, make_layer, make_x
 
@@ -360,8 +558,29 @@ def cpu_baseline(sample_projections: int = 7, repeats: int = 1) -> dict:
         cores = len(os.sched_getaffinity(0))
     except AttributeError:
         cores = os.cpu_count()
-    return {"value": dt * 1e6 / len(shapes), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "decoder-layer copy 0, its %d projections once each, batch 1 (float64: unpack signs, dense W, product)" % len(shapes)}
+    res = {"value": dt * 1e6 / len(shapes), "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": "decoder-layer copy 0, its %d projections once each, batch 1 (float64: unpack signs, dense W, product)" % len(shapes)}
+    if variants:
+        # the same oracle restricted to one thread, and its last step alone (float64 product with W already formed)
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                t0 = time.perf_counter()
+                for L, x in inputs[:2]:
+                    orc.linear(L.planes, L.g, L.h, x)
+                res["one_thread_us_per_layer"] = (time.perf_counter() - t0) * 1e6 / 2
+                res["one_thread_sample"] = "the first two projections (4096 x 4096), BLAS limited to one thread"
+        except ImportError:
+            res["one_thread_us_per_layer"] = None
+        L, x = inputs[0]
+        W = orc.dense_weight(L.planes, L.g, L.h)
+        x64 = x.astype(np.float64)
+        t0 = time.perf_counter()
+        for _ in range(5):
+            (x64 @ W.T)
+        res["w_preformed_us_per_layer"] = (time.perf_counter() - t0) * 1e6 / 5
+        res["w_preformed_sample"] = "4096 x 4096: float64 product alone, dense W formed beforehand by the oracle (not timed)"
+    return res
 
 
 def bench_cases(args) -> dict:
@@ -560,7 +779,7 @@ def bench_trace(args) -> dict:
     torch.cuda.set_device(0)
     device = "cuda:0"
     copies = 3
-    shapes, layers, xs, xs_host, ys = build_workload(copies, 1, device, 16, hints=not args.no_hints)
+    shapes, layers, xs, xs_host, ys = build_workload(copies, 1, device, 16, hints=args.hints)
     lib = binding.raw_lib()
     stream = torch.cuda.Stream(device)
     grouped = not args.no_group
@@ -622,25 +841,46 @@ def bench_trace(args) -> dict:
 
 
 def bench_reference(args) -> dict:
+    """The reference arm: the CPU oracle as it stands, timed on the host cores.  A step is one decoder layer (seven
+    projections); when K steps of the whole layer would not end within a couple of minutes, every step runs the oracle
+    on the first R rows of each projection (rows are independent dot products) and the time is scaled by M / R."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return None
-    per_layer = []
-    base = None
-    for _ in range(max(1, min(args.warmup, 1))):
-        cpu_baseline(sample_projections=1)
+    from oracle import rabit_oracle as orc
+    from synth import llama2_7b_layer_shapes, make_layer, make_x
+    shapes = llama2_7b_layer_shapes()
+    inputs = [(make_layer(sh.M, sh.N, K_PATHS, key=(1, 0, p)), make_x(1, sh.N, key=(1, 10_000))) for p, sh in enumerate(shapes)]
     t0 = time.perf_counter()
-    steps = max(1, min(args.steps, 4))
-    for _ in range(steps):
-        base = cpu_baseline()
-        per_layer.append(base["value"])
-    dt = time.perf_counter() - t0
-    value = float(np.mean(per_layer))
-    base["value"] = value
+    L, x = inputs[0]
+    orc.linear(L.planes[:, :512], L.g[:, :512], L.h, x)                     # warm-up and a cost estimate: 512 rows of 4096 columns
+    est_full_step = (time.perf_counter() - t0) * sum(sh.M * sh.N for sh in shapes) / (512 * 4096)
+    steps = max(1, args.steps)
+    frac = min(1.0, 120.0 / max(est_full_step * (steps + min(args.warmup, 3)), 1e-9))
+    rows = [max(32, int(sh.M * frac) // 32 * 32) for sh in shapes]
+
+    def one_step():
+        t = 0.0
+        for (L, x), sh, R in zip(inputs, shapes, rows):
+            t0 = time.perf_counter()
+            orc.linear(L.planes[:, :R], L.g[:, :R], L.h, x)
+            t += (time.perf_counter() - t0) * sh.M / R
+        return t
+    for _ in range(min(args.warmup, 3)):
+        one_step()
+    per_step = [one_step() for _ in range(steps)]
+    value = float(np.mean(per_step)) * 1e6 / len(shapes)
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count()
+    sample = ("every step: the oracle on the first %s rows of the seven projections of decoder-layer copy 0 (of %s), time scaled to all rows"
+              % ([int(r) for r in rows], [sh.M for sh in shapes]))
+    base = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
     return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
-            "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / steps, "higher_is_better": False,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": float(np.mean(per_step)) * 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": 1, "K": K_PATHS},
+            "config": {"workload": WORKLOAD, "copies": 1, "batch": 1, "K": K_PATHS},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
@@ -648,8 +888,11 @@ def bench_reference(args) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=32000)
-    ap.add_argument("--warmup", type=int, default=640)
+    ap.add_argument("--steps", type=int, default=3200)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--repeats", type=int, default=5, help="timed repeats of the K-step region; value is their median")
+    ap.add_argument("--hints", action="store_true", help="tell every layer which layers run next (weight prefetch across launches)")
+    ap.add_argument("--no-extras", action="store_true", help="only the contract's line: no other configurations, no warm-L2 / read-probe figures")
     ap.add_argument("--impl", default="rabit", choices=["rabit", "reference"])
     ap.add_argument("--copies", type=int, default=32)
     ap.add_argument("--batch", type=int, default=1)
@@ -658,7 +901,6 @@ def main():
     ap.add_argument("--no-group", action="store_true", help="one rabit_linear launch per projection (7 per step instead of 4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-shape", default="", help="extra workloads: keep only the layer shape MxN (e.g. 28672x8192)")
-    ap.add_argument("--no-hints", action="store_true", help="do not tell the layers which layer runs next (no weight prefetch across launches)")
     ap.add_argument("--trace-dump", default="", help="trace7b: also save the raw stamps (numpy file) here")
     ap.add_argument("--workload", default="decoder7b", choices=["decoder7b", "gemm70b", "gemm7b", "gemv70b", "sweep8b", "derive7b", "trace7b"],
                     help="decoder7b is the contract's line; the others are extra single-GPU measurements")

@@ -195,6 +195,16 @@ RABIT_API int rabit_layer_status(const rabit_layer* layer, int clear, void* stre
 RABIT_API int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us, void* stream);
 
 /*
+ * Measurement aid (no counterpart in the paper): one kernel that reads `bytes` bytes of device memory once with
+ * 128-bit streaming loads and keeps nothing.  Timed by the caller with CUDA events over a buffer much larger than L2
+ * it gives the read-only HBM bandwidth this GPU delivers to plain loads, the natural ceiling of the decode GEMV.
+ *   src_dev   DEVICE, 16-byte aligned, `bytes` readable bytes (a multiple of 16 is read)
+ *   sink_dev  DEVICE word or NULL; written only if the data fold to one particular value (keeps the loads alive)
+ * Asynchronous on `stream`.
+ */
+RABIT_API int rabit_selftest_stream_read(const void* src_dev, size_t bytes, unsigned int* sink_dev, void* stream);
+
+/*
  * Host-buffer form of rabit_linear_group: inputs and outputs live in HOST memory (pinned memory makes the
  * copies asynchronous).  An input pointer that occurs several times in xs_host is copied to the device once.
  *   dev_stage  DEVICE, 256-byte aligned, at least rabit_group_stage_bytes(layers, n_layers, batch)

@@ -178,7 +178,6 @@ __device__ __forceinline__ Blk<K> load_blk(const uint4* range_base, int bb, int 
 struct Pending {
     unsigned long long old, add;
     unsigned long long* word;
-    __half* yp;                       // nullptr for padded rows
     bool bad, live;
 };
 
@@ -193,7 +192,8 @@ __device__ __forceinline__ void settle(Pending (&pd)[NB], const LutLayer& L) {
         const long long total = (long long)sum - ((long long)L.n_cs << L.fix_bits);
         const bool poisoned = pd[b].bad || (pd[b].old >> 63) != 0;
         const float v = poisoned ? __int_as_float(0x7FC00000) : __ll2float_rn(total) * L.unit;
-        if (pd[b].yp) *pd[b].yp = __float2half_rn(v);
+        const long long row = (pd[b].word - L.acc) - (long long)b * L.Mp;       // (rare path: the layer's fields come from shared memory)
+        if (row < L.M) L.y[(size_t)b * L.M + row] = __float2half_rn(v);
         *pd[b].word = 0ULL;                                                     // resting state for the next call
     }
 }
@@ -351,9 +351,15 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
     // (the next block's weights, this block's output scales, the atomic adds of the previous block) and its result is
     // first touched below the look-ups of the same iteration, some 1300 cycles later: no request is in flight across the
     // loop's back edge, where the compiler would otherwise have the warp wait for it (a warp has six scoreboards).
+    // what every iteration needs of the layer, in registers (the shared-memory pipe is the one this loop saturates)
+    const unsigned short* const g_base = reinterpret_cast<const unsigned short*>(L.g);
+    unsigned long long* const acc_base = L.acc;
+    const int Mp = L.Mp;
+    const float inv_unit = L.inv_unit, limit = L.limit;
+    const long long bias = (1LL << L.fix_bits) + (1LL << 55);            // shift to non-negative + one arrival
     Pending pd[NB];
 #pragma unroll
-    for (int b = 0; b < NB; ++b) { pd[b].live = false; pd[b].old = 0ULL; pd[b].add = 0ULL; pd[b].word = nullptr; pd[b].yp = nullptr; pd[b].bad = false; }
+    for (int b = 0; b < NB; ++b) { pd[b].live = false; pd[b].old = 0ULL; pd[b].add = 0ULL; pd[b].word = nullptr; pd[b].bad = false; }
     bool owe = false;                                                   // pd holds a finished block whose atomics are still to be issued
     for (int i = 0; i < n_mine; ++i) {
         const int bb = warp + i * kWarps;
@@ -364,7 +370,7 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
         const int row = (seg_rb0 + (bb - seg_begin)) * RABIT_LUT_ROWS + lane;
         unsigned short graw[K];
 #pragma unroll
-        for (int k = 0; k < K; ++k) graw[k] = ldg_u16_early(reinterpret_cast<const unsigned short*>(L.g) + (size_t)k * L.Mp + row);
+        for (int k = 0; k < K; ++k) graw[k] = ldg_u16_early(g_base + (size_t)k * Mp + row);
         Blk<K> nxt = load_blk<K>(range_base, i + 1 < n_mine ? bb + kWarps : bb, lane);   // (the last iteration re-reads its own block: in bounds, unused)
         if (owe) {
 #pragma unroll
@@ -427,12 +433,11 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
             float p = 0.f;
 #pragma unroll
             for (int k = 0; k < K; ++k) p += __half2float(__ushort_as_half(graw[k])) * (acc[b][k][0] + acc[b][k][1]);
-            const float scaled = p * L.inv_unit;
-            const bool bad = !(fabsf(scaled) < L.limit);                  // inf or NaN: finite inputs cannot get here
+            const float scaled = p * inv_unit;
+            const bool bad = !(fabsf(scaled) < limit);                    // inf or NaN: finite inputs cannot get here
             const long long qv = bad ? 0LL : __float2ll_rn(scaled);
-            pd[b].add = (unsigned long long)(qv + (1LL << L.fix_bits)) + (1ULL << 55);
-            pd[b].word = L.acc + (size_t)b * L.Mp + row;
-            pd[b].yp = row < L.M ? L.y + (size_t)b * L.M + row : nullptr;
+            pd[b].add = (unsigned long long)(qv + bias);
+            pd[b].word = acc_base + (size_t)b * Mp + row;
             pd[b].bad = bad;
         }
         owe = true;

@@ -28,7 +28,37 @@ __global__ void bounded_wait_probe(unsigned int* status, long long limit_ns) {
     if (threadIdx.x == 0 && abort_flag) atomicExch(status, 1u);
 }
 
+// Read-only streaming probe: every thread keeps eight 128-bit streaming loads in flight and folds what it reads into
+// one word, which is stored only if it has a value no data here produces (so the loads cannot be dropped).
+__global__ void __launch_bounds__(512) stream_read_probe(const uint4* __restrict__ src, size_t n_vec, unsigned int* sink) {
+    const size_t stride = (size_t)gridDim.x * 512 * 8;
+    uint4 acc = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t base = (size_t)blockIdx.x * 512 * 8 + threadIdx.x; base < n_vec; base += stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const size_t i = base + (size_t)u * 512;
+            v[u] = i < n_vec ? __ldcs(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { acc.x ^= v[u].x; acc.y ^= v[u].y; acc.z ^= v[u].z; acc.w ^= v[u].w; }
+    }
+    if ((acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9E3779B9u && sink) *sink = acc.x;
+}
+
 }  // namespace
+
+extern "C" int rabit_selftest_stream_read(const void* src_dev, size_t bytes, unsigned int* sink_dev, void* stream) {
+    rabit_clear_error();
+    if (!src_dev || ((uintptr_t)src_dev & 15u)) return rabit_fail(RABIT_INVALID_ARG, "rabit_selftest_stream_read: src_dev must be a 16-byte aligned device pointer");
+    if (bytes < 16) return rabit_fail(RABIT_INVALID_ARG, "rabit_selftest_stream_read: bytes must be at least 16");
+    int dev = 0, sms = 0;
+    RABIT_CUDA_TRY(cudaGetDevice(&dev));
+    RABIT_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    stream_read_probe<<<sms * 4, 512, 0, (cudaStream_t)stream>>>((const uint4*)src_dev, bytes / 16, sink_dev);
+    RABIT_CUDA_TRY(cudaGetLastError());
+    return RABIT_OK;
+}
 
 extern "C" int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us, void* stream) {
     rabit_clear_error();
