@@ -114,7 +114,7 @@ def whole_job_us_per_layer(ms_per_step: float, layers_per_step: int, world: int)
 # ---------------------------------------------------------------------------------------
 # workload
 # ---------------------------------------------------------------------------------------
-def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: int = 1, hints: bool = True):
+def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: int = 1):
     import torch
     import paper_2602_05367_b200 as rabit
     from synth import llama2_7b_layer_shapes, make_layer, make_x
@@ -127,17 +127,6 @@ def build_workload(copies: int, batch: int, device: str, tokens: int, seed_cfg: 
             L = make_layer(sh.M, sh.N, K_PATHS, key=(seed_cfg, c, p))
             row.append(rabit.rabit_pack(L.planes, L.g, L.h, device=device))
         layers.append(row)
-    if hints:
-        # the order a decoder runs them in: q|k|v -> o -> gate|up -> down -> the next decoder layer's q|k|v
-        for c in range(copies):
-            nxt = layers[(c + 1) % copies]
-            row = layers[c]
-            for p in (0, 1, 2):
-                row[p].set_next([row[3]])
-            row[3].set_next([row[4], row[5]])
-            row[4].set_next([row[6]])
-            row[5].set_next([row[6]])
-            row[6].set_next([nxt[0], nxt[1], nxt[2]])
     widths = sorted({sh.N for sh in shapes})
     xs_host = {n: np.stack([make_x(batch, n, key=(seed_cfg, 10_000 + t)) for t in range(tokens)]) for n in widths}
     xs = {n: torch.from_numpy(a).to(device) for n, a in xs_host.items()}            # [tokens][batch][N]
@@ -268,7 +257,7 @@ def bench_rabit(args) -> dict:
         torch.cuda.synchronize()
 
     copies, batch, tokens = args.copies, args.batch, 4
-    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens, hints=args.hints)
+    shapes, layers, xs, xs_host, ys = build_workload(copies, batch, device, tokens)
     step_bytes = sum(layer_bytes(sh.M, sh.N, batch) for sh in shapes)
     n_proj = len(shapes)
     stream = torch.cuda.Stream(device)
@@ -389,7 +378,6 @@ def bench_rabit(args) -> dict:
                          "current token are re-read by every layer and stay warm, as in a decoder" % (copies, step_bytes * copies / 1e6),
                    "launch": "CUDA graph replay: the timed region is whole graphs (one graph per cycle over the copies, one for the remainder)",
                    "launches_per_step": launches_per_step,
-                   "next_layer_prefetch_hints": bool(args.hints),
                    "grouping": "q|k|v and gate|up (projections that share their input) each go through one rabit_linear_group launch; "
                                "o and down through rabit_linear" if grouped else "one rabit_linear launch per projection",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -779,7 +767,7 @@ def bench_trace(args) -> dict:
     torch.cuda.set_device(0)
     device = "cuda:0"
     copies = 3
-    shapes, layers, xs, xs_host, ys = build_workload(copies, 1, device, 16, hints=args.hints)
+    shapes, layers, xs, xs_host, ys = build_workload(copies, 1, device, 16)
     lib = binding.raw_lib()
     stream = torch.cuda.Stream(device)
     grouped = not args.no_group
@@ -891,7 +879,6 @@ def main():
     ap.add_argument("--steps", type=int, default=3200)
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--repeats", type=int, default=5, help="timed repeats of the K-step region; value is their median")
-    ap.add_argument("--hints", action="store_true", help="tell every layer which layers run next (weight prefetch across launches)")
     ap.add_argument("--no-extras", action="store_true", help="only the contract's line: no other configurations, no warm-L2 / read-probe figures")
     ap.add_argument("--impl", default="rabit", choices=["rabit", "reference"])
     ap.add_argument("--copies", type=int, default=32)

@@ -254,18 +254,6 @@ RABIT_API int rabit_layer_N(const rabit_layer* layer);
  */
 RABIT_API int rabit_set_variant(rabit_layer* layer, int variant);
 
-/*
- * Prefetch hint for decode chains (no counterpart in the paper; the layer's result does not change).  Names up to 8
- * layers that the caller will run right after `layer` (for a decoder: q|k|v -> o -> gate|up -> down -> the next
- * block's q|k|v).  From then on the batch 1..2 kernel of `layer` (alone or inside a group) asks L2, at its very
- * start, to fetch the look-up blocks of those layers, so that they cross HBM - and their pages enter the TLBs -
- * while this kernel still waits for its input and computes, instead of at the start of their own kernel, which at
- * a few microseconds per layer would otherwise begin with an idle HBM and a memory latency on its critical path.
- * Every byte still crosses HBM once.  n_next = 0 removes the hint.  The device buffers of the named layers must
- * stay allocated for as long as the hint is set (freeing their descriptors is fine; the hint keeps addresses).
- */
-RABIT_API int rabit_set_next(rabit_layer* layer, const rabit_layer* const* next, int n_next);
-
 /* Release the descriptor only; the caller's device buffer is untouched. NULL is accepted. */
 RABIT_API int rabit_free(rabit_layer* layer);
 

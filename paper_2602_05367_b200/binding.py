@@ -69,8 +69,6 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = [_c_void_p]
     lib.rabit_set_variant.restype = _c_int
     lib.rabit_set_variant.argtypes = [_c_void_p, _c_int]
-    lib.rabit_set_next.restype = _c_int
-    lib.rabit_set_next.argtypes = [_c_void_p, _c_void_p, _c_int]
     lib.rabit_free.restype = _c_int
     lib.rabit_free.argtypes = [_c_void_p]
     lib.rabit_trace_begin.restype = _c_int
@@ -165,14 +163,6 @@ class RabitLayer:
         5 table-driven GEMV."""
         _check(_lib.rabit_set_variant(self.handle, variant))
 
-    def set_next(self, next_layers) -> None:
-        """Prefetch hint: the layers that will run right after this one (up to 8; an empty list removes the hint).
-        The named layers' device buffers must stay alive while the hint is set."""
-        n = len(next_layers)
-        arr = (_c_void_p * max(n, 1))(*[l.handle for l in next_layers])
-        _check(_lib.rabit_set_next(self.handle, arr, n))
-        self._next_keepalive = [l.dev_buf for l in next_layers]
-
     def status(self, clear: bool = False, stream: int = 0) -> int:
         """0 if every kernel of this layer completed its waits, RABIT_DEVICE_FAULT (-5) otherwise; synchronises."""
         return int(_lib.rabit_layer_status(self.handle, 1 if clear else 0, _c_void_p(stream)))
@@ -190,7 +180,6 @@ class RabitLayer:
             self._handle = None
             self.dev_buf = None
             self._stage = None
-            self._next_keepalive = None
 
     def __del__(self):  # pragma: no cover
         try:

@@ -36,7 +36,6 @@ static void bind_layer(rabit_layer* L, const RabitGeom& G, const RabitHeader& hd
     L->d_status = L->d_flags + ((size_t)G.n_rt * G.K + RABIT_MAX_GRID);
     L->d_lut = (const unsigned char*)(L->dev_base + hdr.off_lut);
     L->d_acc = (unsigned long long*)(L->dev_base + hdr.off_acc);
-    L->n_next = 0;
 }
 
 extern "C" int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
@@ -476,23 +475,6 @@ extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
     if (variant < 0 || variant > 5) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..5");
     layer->variant = variant;
-    return RABIT_OK;
-}
-
-extern "C" int rabit_set_next(rabit_layer* layer, const rabit_layer* const* next, int n_next) {
-    rabit_clear_error();
-    if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: layer is NULL");
-    if (n_next < 0 || n_next > 8) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: n_next must be 0..8 (got %d)", n_next);
-    if (n_next > 0 && !next) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: next is NULL");
-    for (int s = 0; s < n_next; ++s) {
-        if (!next[s]) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: null entry %d", s);
-        if (next[s]->device != layer->device) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_next: entry %d lives on another device", s);
-    }
-    layer->n_next = n_next;
-    for (int s = 0; s < n_next; ++s) {
-        layer->next_ptr[s] = next[s]->d_lut;
-        layer->next_bytes[s] = (unsigned long long)next[s]->geom.n_cs * next[s]->geom.n_rb * next[s]->geom.K * RABIT_LUT_PART_BYTES;
-    }
     return RABIT_OK;
 }
 

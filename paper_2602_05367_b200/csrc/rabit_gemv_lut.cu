@@ -17,13 +17,14 @@
 // the same: so much per block, so much per table), which is one contiguous byte range.  A range that
 // crosses into the next 256-column slice rebuilds its table there.  One CTA per SM, 16 warps:
 //   * before the dependency wait (weights do not depend on the previous kernel in the stream, so this
-//     overlaps its tail under programmatic dependent launch): one thread asks for the CTA's whole byte
-//     range to be prefetched into L2 (bulk prefetch, 64 KB per instruction), every warp loads its first
-//     block into registers, and the input scales of the first table are read;
+//     overlaps its tail under programmatic dependent launch): every warp loads its first block into
+//     registers and the input scales of the first table are read (a bulk L2 prefetch of the CTA's whole
+//     range at this point was measured and made the kernel 8-10 % slower: the loads then meet their own
+//     prefetch in L2);
 //   * after the wait: x of the slice is read, the table is built (lane = byte group, warp = path x upper
 //     three index bits; 32 entries each by doubling), and the warps take the blocks round-robin, lane =
 //     row.  A lane holds its 16*K weight words in registers (128-bit streaming loads, one block ahead:
-//     32 KB in flight per SM, on top of the L2 prefetch), walks the 32 byte groups of
+//     32 KB in flight per SM; two ahead measured no faster), walks the 32 byte groups of
 //     its row in an order rotated by its lane index (so the 32 look-ups of a warp step hit 32 banks), and
 //     ends with  p = sum_k g_k[row] * s_k;
 //   * reduction over the slices of a row, without a second pass, a fence or a wait: p is rounded to a
@@ -48,8 +49,6 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kMaxGrid = 160;
 constexpr int kMaxGroup = 8;
 constexpr unsigned long long kSumMask = (1ULL << 55) - 1;
-constexpr unsigned int kPrefetchChunk = 65536;            // bytes per L2 bulk prefetch instruction
-constexpr long long kPrefetchMax = 1 << 20;               // most bytes a CTA asks to be prefetched
 
 // Tables: one 64 KB table serves two paths, entry e of (path k, byte group) at  e * 256 + (k & 1) * 128 + group * 4
 // of table k >> 1.  The tables start on a 64 KB boundary of the CTA's shared-memory window, so that a table address
@@ -88,10 +87,6 @@ struct CtaRange {
 };
 struct LutParams {
     int n_layers;
-    int n_next;                     // successor layers whose look-up blocks this launch asks L2 to fetch (hint)
-    const unsigned char* next_ptr[kMaxGroup];
-    unsigned int next_bytes[kMaxGroup];   // per CTA: CTA c prefetches [c * next_bytes, (c + 1) * next_bytes) of successor s, clipped to next_total
-    unsigned long long next_total[kMaxGroup];
     unsigned long long* trace;      // RABIT_TRACE builds: 8 time stamps per CTA of this launch (nullptr: none)
     LutLayer layer[kMaxGroup];
     CtaRange range[kMaxGrid];
@@ -135,9 +130,6 @@ __device__ __forceinline__ unsigned long long use_here_u64(unsigned long long v)
     unsigned long long r;
     asm volatile("mov.b64 %0, %1;" : "=l"(r) : "l"(v));
     return r;
-}
-__device__ __forceinline__ void prefetch_l2(const void* p, unsigned int bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 // Phase stamps of a CTA (RABIT_TRACE builds only; see rabit_trace_begin in rabit.h): stamp 0 is %globaltimer
@@ -230,24 +222,6 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
     const uint4* range_base = reinterpret_cast<const uint4*>(range_bytes);
 
     // ---- everything that does not depend on the stream's past
-    if (tid == 0) {
-        long long left = (long long)n_blocks * (K * RABIT_LUT_PART_BYTES);
-        if (left > kPrefetchMax) left = kPrefetchMax;
-        for (long long off = 0; off < left; off += kPrefetchChunk)
-            prefetch_l2(range_bytes + off, (unsigned int)(left - off < kPrefetchChunk ? left - off : kPrefetchChunk));
-    }
-    if (tid == 32) {
-        // the layers the caller named as the next ones to run: their weights cross HBM (and their pages enter the
-        // TLBs) while this kernel waits and computes, instead of at the start of their own kernel
-        for (int s = 0; s < P.n_next; ++s) {
-            const unsigned long long lo = (unsigned long long)blockIdx.x * P.next_bytes[s];
-            if (lo >= P.next_total[s]) continue;
-            unsigned long long left = P.next_total[s] - lo;
-            if (left > P.next_bytes[s]) left = P.next_bytes[s];
-            for (unsigned long long off = 0; off < left; off += kPrefetchChunk)
-                prefetch_l2(P.next_ptr[s] + lo + off, (unsigned int)(left - off < kPrefetchChunk ? left - off : kPrefetchChunk));
-        }
-    }
     const int n_mine = warp < n_blocks ? (n_blocks - warp + kWarps - 1) / kWarps : 0;    // blocks warp, warp + 16, ...
     Blk<K> cur;                                          // this warp's current block
 #pragma unroll
@@ -637,22 +611,6 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
     const int launch_grid = c0;
     for (int i = c0; i < kMaxGrid; ++i) P.range[i] = CtaRange{0, 0, 0};
     const int device = layers[0]->device;
-    // successors named by rabit_set_next on any layer of the group (each once)
-    P.n_next = 0;
-    for (int l = 0; l < n_layers; ++l)
-        for (int s = 0; s < layers[l]->n_next && P.n_next < kMaxGroup; ++s) {
-            bool seen = false;
-            for (int t = 0; t < P.n_next; ++t) seen = seen || P.next_ptr[t] == layers[l]->next_ptr[s];
-            if (seen || layers[l]->next_bytes[s] == 0) continue;
-            const unsigned long long total = layers[l]->next_bytes[s];
-            unsigned long long per_cta = (total + launch_grid - 1) / launch_grid;
-            per_cta = (per_cta + 1023) & ~1023ULL;                       // whole 1 KB parts (16-byte granularity is what the instruction needs)
-            P.next_ptr[P.n_next] = layers[l]->next_ptr[s];
-            P.next_bytes[P.n_next] = (unsigned int)per_cta;
-            P.next_total[P.n_next] = total;
-            ++P.n_next;
-        }
-    for (int s = P.n_next; s < kMaxGroup; ++s) { P.next_ptr[s] = nullptr; P.next_bytes[s] = 0; P.next_total[s] = 0; }
     P.trace = rabit_trace_slot(launch_grid);
     if (K == 1) return batch == 1 ? launch_inst<1, 1>(P, launch_grid, device, stream) : launch_inst<1, 2>(P, launch_grid, device, stream);
     if (K == 2) return batch == 1 ? launch_inst<2, 1>(P, launch_grid, device, stream) : launch_inst<2, 2>(P, launch_grid, device, stream);

@@ -24,9 +24,6 @@ struct rabit_layer {
     unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
     const unsigned char* d_lut;  // look-up blocks (table-driven GEMV)
     unsigned long long* d_acc;   // u64 [RABIT_LUT_MAX_BATCH][Mp] accumulate words of the table-driven GEMV (zero between calls)
-    int n_next;                  // rabit_set_next: look-up sections the decode kernel of this layer asks L2 to fetch
-    const unsigned char* next_ptr[8];
-    unsigned long long next_bytes[8];
 };
 
 // error reporting (thread-local message); returns `code`
