@@ -83,8 +83,10 @@ RABIT_API int rabit_unpack_host(const void* image, size_t image_bytes,
  *                     valid and unmodified by the caller until rabit_free.
  *   stream    the copy is enqueued on it and the call returns after it has completed.
  *   out       receives the new descriptor.
- * The reduction scratch inside dev_buf starts zeroed and is left zeroed by every call of
- * rabit_linear, so calls on one layer must not overlap in time (different layers may).
+ * dev_buf also holds the layer's reduction scratch, in its resting state: the fp32 exchange buffer of the tensor-core
+ * GEMV is all-ones words (0xFFFFFFFF, "nothing published"), the 64-bit accumulate words of the table-driven GEMV, the
+ * reserved flags and the status word are zero.  Every call leaves it in that state, so calls on one layer must not
+ * overlap in time (different layers may).  A caller that moves or restores an image must keep these values.
  */
 RABIT_API int rabit_pack(const uint32_t* planes, const uint16_t* g, const uint16_t* h,
                int K, int M, int N, void* dev_buf, size_t dev_bytes, void* stream,
@@ -174,15 +176,24 @@ RABIT_API int rabit_linear_host(const rabit_layer* layer, const void* x_host, vo
  *     layer uses back into its resting state (memsets enqueued on `stream` ahead of the kernel).  Two calls that overlap on the
  *     GPU (different streams, or one stream per thread) race on it and give wrong results: keep
  *     all uses of this entry point on one stream, or serialise them yourself.
- * Results equal those of rabit_linear (same kernel, same summation order).
+ *   - This entry point always runs the integer tensor-core GEMV (the kernel whose scratch is large enough to matter);
+ *     rabit_linear may choose another kernel for the same call, so the two agree within the parity tolerance, not bit
+ *     for bit.  A bounded wait that runs out in it is recorded in a status word inside the array, which
+ *     rabit_layer_status reports (for any layer of that device) and clears.
  */
 RABIT_API int rabit_linear_static_scratch(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
 /*
  * Health of a layer's kernels.  Every wait inside the kernels is bounded (about one second); a wait that
- * runs out makes the kernel set the layer's status word, skip its remaining waits and return, so the
- * context stays usable but the outputs of that call are invalid.  This call synchronises `stream`, reads
- * the word and returns RABIT_OK or RABIT_DEVICE_FAULT (the word is cleared when `clear` is non-zero).
+ * runs out makes the kernel set a status word, skip its remaining waits and return, so the context stays
+ * usable but the outputs of that call are invalid.  (Only the tensor-core kernels wait for anything: the GEMV for
+ * bulk copies and for the partial sums of CTAs with a lower index - it assumes that the CTAs of a grid no larger
+ * than the device holds at once all become resident while it waits, which another tenant on the GPU can delay
+ * beyond the limit - and the GEMM for its copy and tensor-memory barriers.  The table-driven GEMV never waits.)
+ * A grouped launch records a run-out wait in the status word of every layer of the group.
+ * This call synchronises `stream`, reads the layer's word and the word of the built-in scratch array of
+ * rabit_linear_static_scratch, and returns RABIT_OK or RABIT_DEVICE_FAULT.  With `clear` non-zero it also puts the
+ * words and the layer's exchange buffer back into their resting state; do that before the layer is used again.
  */
 RABIT_API int rabit_layer_status(const rabit_layer* layer, int clear, void* stream);
 

@@ -163,8 +163,11 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
 
     int variant = layer->variant;
     if (variant == 0) {
+        const double packed_mb = (double)G.K * G.Mp * G.N / 8.0e6;
         if (rabit_gemv_lut_supports(*layer, batch)) {
             variant = 5;
+        } else if (batch <= 4 && packed_mb <= 8.0 && rabit_gemv_lut_supports(*layer, 1)) {
+            variant = 5;                    // two passes of the table-driven kernel: measured faster than one pass of the tensor-core GEMV on small layers
         } else if (batch <= RABIT_MAX_GEMV_BATCH) {
             variant = rabit_gemv_mma_supports(*layer, batch) ? 2 : 1;
             // From 5 batch rows on the GEMV makes two to four passes over the weights; the tensor-core GEMM, whose cost
@@ -389,15 +392,25 @@ extern "C" int rabit_layer_status(const rabit_layer* layer, int clear, void* str
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_layer_status: layer is NULL");
     cudaStream_t st = (cudaStream_t)stream;
-    unsigned int word = 0;
+    // two words can record a wait that ran out: the layer's own (inside its packed image) and the one of the library's
+    // built-in scratch array, which rabit_linear_static_scratch uses for every layer
+    unsigned int word = 0, word_static = 0;
+    unsigned int* d_static = rabit_static_scratch_status(layer->device);
     RABIT_CUDA_TRY(cudaMemcpyAsync(&word, layer->d_status, 4, cudaMemcpyDeviceToHost, st));
+    if (d_static) RABIT_CUDA_TRY(cudaMemcpyAsync(&word_static, d_static, 4, cudaMemcpyDeviceToHost, st));
     RABIT_CUDA_TRY(cudaStreamSynchronize(st));
-    if (word != 0) {
+    if (word != 0 || word_static != 0) {
         if (clear) {
+            // a contributor that gave up may still have published a partial sum after its finisher restored the resting
+            // state: put the whole exchange buffer back, not just the word
+            const size_t partial_bytes = (size_t)((const char*)layer->d_flags - (const char*)layer->d_partial);
+            RABIT_CUDA_TRY(cudaMemsetAsync(layer->d_partial, 0xFF, partial_bytes, st));
             RABIT_CUDA_TRY(cudaMemsetAsync(layer->d_status, 0, 4, st));
+            if (d_static) RABIT_CUDA_TRY(cudaMemsetAsync(d_static, 0, 4, st));
             RABIT_CUDA_TRY(cudaStreamSynchronize(st));
         }
-        return rabit_fail(RABIT_DEVICE_FAULT, "rabit_layer_status: a kernel of this layer gave up on a bounded wait; its outputs are invalid");
+        return rabit_fail(RABIT_DEVICE_FAULT, "rabit_layer_status: a kernel of this layer%s gave up on a bounded wait; the outputs of that call are invalid",
+                          word_static != 0 ? " (or another layer run through the built-in scratch array)" : "");
     }
     return RABIT_OK;
 }

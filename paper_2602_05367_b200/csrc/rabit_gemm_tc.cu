@@ -562,18 +562,19 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
     P.batch = batch;
     P.n_bt = (batch + TB - 1) / TB;
     const int n_tiles = L.geom.n_rt * P.n_bt;
-    static bool attr_done = false;
+    static bool attr_done[64] = {false};                                          // function attributes are per device
+    const int dev_slot = L.device >= 0 && L.device < 64 ? L.device : 0;
     const size_t smem = sizeof(Smem<TB, KP, DEQ ? 1 : KP>) + 1024;               // slack for the 1024-byte alignment of the stages
-    if (!attr_done) {
+    if (!attr_done[dev_slot] || dev_slot != L.device) {
         cudaError_t e = cudaFuncSetAttribute(rabit_gemm_tc_kernel<TB, KP, DEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done[dev_slot] = true;
     }
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
     const bool ring_holds_exchange = sizeof(InStage<TB, KP>) * GemmCfg<TB, KP, DEQ ? 1 : KP>::kStages >= (size_t)kTileM * TB * 4;   // the receive buffer lives in the input ring
 
-    static bool limits_done = false;
-    if (!limits_done) {                                            // how many clusters of each size fit at once (asked once per kernel)
+    static bool limits_done[64] = {false};
+    if (!limits_done[dev_slot]) {                                            // how many clusters of each size fit at once (asked once per kernel)
         for (int lg = 1; lg <= 3; ++lg) {
             cudaLaunchConfig_t q = {};
             q.gridDim = dim3((unsigned int)((sms / (1 << lg)) * (1 << lg)));
@@ -590,7 +591,7 @@ static cudaError_t launch_gemm(const rabit_layer& L, const void* x, void* y, int
             if (cudaOccupancyMaxActiveClusters(&n, rabit_gemm_tc_kernel<TB, KP, DEQ>, &q) == cudaSuccess && n > 0) g_cluster_limit[lg] = n;
             else cudaGetLastError();
         }
-        limits_done = true;
+        limits_done[dev_slot] = true;
     }
 
     // One launch over tiles [lo, hi).  Few tiles: the CTAs of a cluster share each tile's contraction (see choose_split).

@@ -37,6 +37,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstring>
 #include <type_traits>
 #include <vector>
 
@@ -438,7 +439,9 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
 struct Cost {
     long long block, table;
 };
-Cost cost_of(int K, int nb) { return Cost{(long long)nb * (40 * K + 10), (long long)nb * (260 * K) + 200}; }
+// SM clock cycles, from the phase stamps of the kernel on B200: a block of K paths (look-ups, loads, its atomic) and a
+// table (build plus the two barriers around it).
+Cost cost_of(int K, int nb) { return Cost{(long long)nb * (70 * K + 30), (long long)nb * (200 * K) + 100}; }
 
 // CTAs a layer of n_cs x n_rb blocks needs when no CTA may cost more than `limit`; writes the cuts if asked.
 int ctas_needed(int n_cs, int n_rb, const Cost& C, long long limit, std::vector<int>* cuts) {
@@ -499,6 +502,12 @@ cudaError_t launch_inst(const LutParams& P, int grid, int device, cudaStream_t s
     return cudaLaunchKernelEx(&cfg, rabit_gemv_lut_kernel<K, NB>, P);
 }
 
+cudaError_t launch_k(int K, int batch, const LutParams& P, int grid, int device, cudaStream_t stream) {
+    if (K == 1) return batch == 1 ? launch_inst<1, 1>(P, grid, device, stream) : launch_inst<1, 2>(P, grid, device, stream);
+    if (K == 2) return batch == 1 ? launch_inst<2, 1>(P, grid, device, stream) : launch_inst<2, 2>(P, grid, device, stream);
+    return launch_inst<3, 1>(P, grid, device, stream);
+}
+
 }  // namespace
 
 int rabit_gemv_lut_max_rows() { return 2; }
@@ -552,6 +561,21 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
         total_blocks += blocks;
     }
     for (int l = n_layers; l < kMaxGroup; ++l) P.layer[l] = P.layer[0];
+    // The cut of the layers into ranges depends only on the shapes, the batch and the device: remembered per thread
+    // (a decoder calls the same few groups over and over; the search costs a few microseconds of host time).
+    struct PlanKey { int n, batch, sms, shape[kMaxGroup][3]; };
+    struct Plan { PlanKey key; int grid; CtaRange range[kMaxGrid]; };
+    static thread_local std::vector<Plan> plans;
+    PlanKey key;
+    std::memset(&key, 0, sizeof(key));
+    key.n = n_layers; key.batch = batch; key.sms = layers[0]->sm_count;
+    for (int l = 0; l < n_layers; ++l) { key.shape[l][0] = K; key.shape[l][1] = layers[l]->geom.n_rb; key.shape[l][2] = layers[l]->geom.n_cs; }
+    for (const Plan& pl : plans)
+        if (std::memcmp(&pl.key, &key, sizeof(key)) == 0) {
+            std::memcpy(P.range, pl.range, sizeof(P.range));
+            P.trace = rabit_trace_slot(pl.grid);
+            return launch_k(K, batch, P, pl.grid, layers[0]->device, stream);
+        }
     int sms = layers[0]->sm_count > 0 ? layers[0]->sm_count : 148;
     int grid = sms < kMaxGrid ? sms : kMaxGrid;
     if ((long long)grid > total_blocks) grid = (int)total_blocks;
@@ -610,11 +634,13 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
     }
     const int launch_grid = c0;
     for (int i = c0; i < kMaxGrid; ++i) P.range[i] = CtaRange{0, 0, 0};
-    const int device = layers[0]->device;
+    if (plans.size() >= 256) plans.clear();
+    plans.emplace_back();
+    plans.back().key = key;
+    plans.back().grid = launch_grid;
+    std::memcpy(plans.back().range, P.range, sizeof(P.range));
     P.trace = rabit_trace_slot(launch_grid);
-    if (K == 1) return batch == 1 ? launch_inst<1, 1>(P, launch_grid, device, stream) : launch_inst<1, 2>(P, launch_grid, device, stream);
-    if (K == 2) return batch == 1 ? launch_inst<2, 1>(P, launch_grid, device, stream) : launch_inst<2, 2>(P, launch_grid, device, stream);
-    return launch_inst<3, 1>(P, launch_grid, device, stream);
+    return launch_k(K, batch, P, launch_grid, layers[0]->device, stream);
 }
 
 cudaError_t rabit_launch_gemv_lut(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {

@@ -1,4 +1,5 @@
-// Decode GEMV on the integer tensor-core path (batch 1..2 per launch).
+// Decode GEMV on the integer tensor-core path (1, 2 or 4 batch rows per launch; the dispatcher uses it for batches
+// 3..16, the table-driven kernel of rabit_gemv_lut.cu takes batches 1..2).
 //
 //   y[b][i] = sum_k g_k[i] * sum_j B_k[i][j] * t_k[b][j],   t_k[b][j] = h_k[j] * x[b][j]     (Section 4.1, Eq. 2)
 //
@@ -8,14 +9,15 @@
 // packed word masked with 0x01010101 << p is already a u8 MMA operand with entries {0, 2^p}
 // (see rabit_layout.h), and mma.sync.m16n8k32.u8.s8 does the additions.  The B operand holds
 // t in exact fixed point: T = round(t * sigma), sigma a power of two chosen per (path,
-// batch row) from max|x| * max|h_k| so that |T| < 2^30, split into four balanced base-256
+// batch row) from max|x| * max|h_k| so that |T| < 2^28, split into four balanced base-256
 // digits that occupy four of the eight MMA columns (a second batch row takes the other
 // four).  With b the sign bit, sum_j B t = sum_j t - 2 sum_j b t; the int32 accumulators
 // give sum_j b T per digit exactly, and the epilogue recombines the digits, applies
-// 1/sigma, g_k and the path sum in fp32.  The roundings are T (at most 2^-31 of the bound
+// 1/sigma, g_k and the path sum in fp32.  The roundings are T (at most 2^-29 of the bound
 // per term), the fp32 epilogue and the final fp16 store.
 //
-// Structure of a CTA (10 warps, two CTAs per SM):
+// Structure of a CTA (8 MMA warps plus 2 builder warps and two CTAs per SM up to two batch rows; 4 builder warps and
+// one CTA per SM at four):
 //   * The tiles of the layer are numbered in layout order; CTA c owns positions
 //     [c*T/G, (c+1)*T/G), one contiguous byte range, so the split is even for every shape.
 //   * One elected thread streams that range with bulk asynchronous copies into a ring of
@@ -32,7 +34,11 @@
 //     ones, a NaN no arithmetic here produces): the data is its own "published" flag.  The
 //     CTA that owns the last tile of a row tile finishes it: each of its threads reads the
 //     partials of its row from the other contributors (all of them CTAs with a lower index,
-//     so the waits cannot form a cycle), waiting (bounded) while it still sees the sentinel,
+//     so the waits cannot form a cycle as long as those CTAs are resident or become resident while it
+//     waits: the grid is never larger than what the device holds at once, but CUDA does not promise the
+//     order in which CTAs start, and another kernel or tenant on the GPU can delay them; the wait is
+//     bounded, so that case ends as a recorded time-out with invalid outputs, not as a hang), waiting
+//     (bounded) while it still sees the sentinel,
 //     puts the sentinel back, adds in a fixed order (deterministic) and stores fp16.
 // Every wait in the kernel is bounded; a wait that runs out sets a status word and the
 // kernel drains and returns (results are then invalid, the context stays usable).
@@ -102,7 +108,7 @@ struct GemvParams {
 constexpr int kMaxGroup = 8;
 struct GroupParams {
     int n_layers;
-    unsigned int* status;
+    unsigned int* status[kMaxGroup];   // the status word of every layer of the group: a wait that runs out is recorded in all of them
     int nb;                  // batch rows actually present (<= the kernel's NB); the others are neither read nor written
     GemvParams layer[kMaxGroup];
 };
@@ -672,7 +678,7 @@ rabit_gemv_mma_kernel(const __grid_constant__ GroupParams GP) {
             while (!mbar_try_wait(smem_u32(&S.full[it % kRing]), (it / kRing) & 1))
                 if (clock64() - t0 > kWaitLimitCycles) break;
         }
-        atomicExch(GP.status, 1u);
+        for (int l = 0; l < GP.n_layers; ++l) atomicExch(GP.status[l], 1u);
     }
 }
 
@@ -684,13 +690,14 @@ bool rabit_gemv_mma_supports(const rabit_layer& L, int batch) {
 }
 
 template <int NB>
-static cudaError_t launch_nb(const GroupParams& GP, int grid, cudaStream_t stream) {
-    static bool attr_done = false;
+static cudaError_t launch_nb(const GroupParams& GP, int grid, int device, cudaStream_t stream) {
+    static bool attr_done[64] = {false};                                          // function attributes are per device
+    const int dev_slot = device >= 0 && device < 64 ? device : 0;
     const size_t smem = sizeof(Smem<NB>);
-    if (!attr_done) {
+    if (!attr_done[dev_slot] || dev_slot != device) {
         cudaError_t e = cudaFuncSetAttribute(rabit_gemv_mma_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done[dev_slot] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -723,7 +730,7 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
     if (batch < 1 || batch > 4) return cudaErrorInvalidValue;
     GroupParams GP;
     GP.n_layers = n_layers;
-    GP.status = layers[0]->d_status;
+    for (int l = 0; l < kMaxGroup; ++l) GP.status[l] = layers[l < n_layers ? l : 0]->d_status;
     GP.nb = batch;
     long long total = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -785,9 +792,10 @@ cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_
     }
     for (int l = n_layers; l < kMaxGroup; ++l) { GP.layer[l] = GP.layer[0]; GP.layer[l].n_cta = 0; }
     const int launch_grid = c0;
-    if (batch == 1) return launch_nb<1>(GP, launch_grid, stream);
-    if (batch == 2) return launch_nb<2>(GP, launch_grid, stream);
-    return launch_nb<4>(GP, launch_grid, stream);
+    const int device = layers[0]->device;
+    if (batch == 1) return launch_nb<1>(GP, launch_grid, device, stream);
+    if (batch == 2) return launch_nb<2>(GP, launch_grid, device, stream);
+    return launch_nb<4>(GP, launch_grid, device, stream);
 }
 
 cudaError_t rabit_launch_gemv_mma(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream) {

@@ -20,7 +20,7 @@ struct rabit_layer {
     const uint16_t* d_g;         // fp16 [K][Mp]
     const uint16_t* d_h;         // fp16 [K][N]
     float* d_partial;            // fp32 [n_rt*K + RABIT_MAX_GRID][RABIT_PARTIAL_BATCH][128] cross-CTA partial sums (all-ones words between calls)
-    unsigned int* d_flags;       // u32 [n_rt*K + RABIT_MAX_GRID] reserved (zero), then one status word
+    unsigned int* d_flags;       // u32 [n_rt*K + RABIT_MAX_GRID] reserved (stay zero; no kernel uses them), then one status word
     unsigned int* d_status;      // u32, non-zero once a kernel gave up on a bounded wait
     const unsigned char* d_lut;  // look-up blocks (table-driven GEMV)
     unsigned long long* d_acc;   // u64 [RABIT_LUT_MAX_BATCH][Mp] accumulate words of the table-driven GEMV (zero between calls)
@@ -62,6 +62,8 @@ int rabit_gemv_mma_max_rows();
 bool rabit_gemv_mma_group_supports(const rabit_layer* const* layers, int n_layers, int batch);
 cudaError_t rabit_launch_gemv_mma_group(const rabit_layer* const* layers, int n_layers, const void* const* xs, void* const* ys,
                                         int batch, cudaStream_t stream);
+unsigned int* rabit_static_scratch_status(int device);   // rabit_noalloc.cu; nullptr before the first static-scratch call on that device
+
 // Phase tracing (rabit_api.cu): the next free record of 8 stamps x `ctas` in the caller's trace buffer, or nullptr
 // when tracing is off, the buffer is full or the library was built without RABIT_TRACE.
 unsigned long long* rabit_trace_slot(int ctas);

@@ -13,6 +13,8 @@ namespace {
 
 constexpr size_t kScratchBytes = (size_t)4 << 20;        // 4 MiB, held by every GPU that loads the library
 constexpr int kMaxDevices = 64;
+constexpr size_t kStatusOffset = kScratchBytes - 256;    // one status word for all calls, at a fixed place; it starts at zero
+                                                         // (static storage) and only rabit_layer_status(clear) puts it back
 
 // Partial sums | reserved | status word.  Every call shares this array.
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
@@ -32,11 +34,17 @@ ScratchPlan plan_for(const RabitGeom& G) {
     p.flags_off = rabit_align256(p.partial_bytes);
     p.flags_bytes = p.entries * 4;
     p.status_off = p.flags_off + rabit_align256(p.flags_bytes);
-    p.total = p.status_off + 256;
+    p.total = p.status_off + 256;                            // (the status word itself sits at the end of the array, see kStatusOffset)
     return p;
 }
 
 }  // namespace
+
+// The status word of the built-in array on `device`, or nullptr if no call has set the array up there yet.
+unsigned int* rabit_static_scratch_status(int device) {
+    if (device < 0 || device >= kMaxDevices || !g_scratch_ptr[device]) return nullptr;
+    return reinterpret_cast<unsigned int*>(g_scratch_ptr[device] + kStatusOffset);
+}
 
 extern "C" int rabit_linear_static_scratch(const rabit_layer* layer, const void* x, void* y, int batch, void* stream) {
     rabit_clear_error();
@@ -55,7 +63,7 @@ extern "C" int rabit_linear_static_scratch(const rabit_layer* layer, const void*
     if (!rabit_gemv_mma_supports(*layer, batch))
         return rabit_fail(RABIT_UNSUPPORTED_SHAPE, "rabit_linear_static_scratch: the GEMV kernel cannot run this layer");
     const ScratchPlan plan = plan_for(G);
-    if (plan.total > kScratchBytes)
+    if (plan.total > kStatusOffset)
         return rabit_fail(RABIT_UNSUPPORTED_SHAPE,
                           "rabit_linear_static_scratch: layer needs %zu bytes of reduction scratch, the built-in array holds %zu "
                           "(K * ceil(M/128) must stay below about %zu)",
@@ -77,12 +85,12 @@ extern "C" int rabit_linear_static_scratch(const rabit_layer* layer, const void*
     // The array keeps whatever the last call (of any layer) left: the partial slots of this layer must
     // start in their resting state (all-ones words) and the status word at zero.
     RABIT_CUDA_TRY(cudaMemsetAsync(base, 0xFF, plan.partial_bytes, st));
-    RABIT_CUDA_TRY(cudaMemsetAsync(base + plan.flags_off, 0, plan.status_off + 256 - plan.flags_off, st));
+    RABIT_CUDA_TRY(cudaMemsetAsync(base + plan.flags_off, 0, plan.status_off - plan.flags_off, st));
 
     rabit_layer view = *layer;                               // same weights and scales, scratch redirected
     view.d_partial = reinterpret_cast<float*>(base);
     view.d_flags = reinterpret_cast<unsigned int*>(base + plan.flags_off);
-    view.d_status = reinterpret_cast<unsigned int*>(base + plan.status_off);
+    view.d_status = reinterpret_cast<unsigned int*>(base + kStatusOffset);
     cudaError_t e = cudaSuccess;
     const int rows = rabit_gemv_mma_max_rows();
     for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += rows)

@@ -77,22 +77,21 @@ def test_gemm_runs_small_batches_too(K, M, N, batch):
 
 @pytest.mark.parametrize("batch", [4, 8, 12, 16])
 def test_dispatch_between_five_and_sixteen_rows(batch):
-    """Up to four batch rows always take the GEMV (one pass); beyond that the dispatcher compares its cost estimates of
-    the GEMV passes and of one GEMM launch.  Whichever kernel runs, the result is within tolerance and is exactly what
-    that kernel gives when forced; on this tall, narrow layer 16 rows go to the GEMM."""
+    """Up to four batch rows take a decode GEMV (table-driven passes of two rows on small layers, else one pass of the
+    tensor-core GEMV); beyond that the dispatcher compares its cost estimates of the GEMV passes and of one GEMM launch.
+    Whichever kernel runs, the result is within tolerance and is exactly what that kernel gives when forced; on this tall,
+    narrow layer 16 rows go to the GEMM."""
     L = make_layer(14336, 512, 2, key=(63,))
     x = make_x(batch, 512, key=(63, batch))
     y_auto = run_layer(L, x, 0)
     check_against_oracle(L, x, y_auto)
-    y_gemv = run_layer(L, x, 2)
-    y_gemm = run_layer(L, x, GEMM)
-    same_gemv = np.array_equal(y_auto.view(np.uint16), y_gemv.view(np.uint16))
-    same_gemm = np.array_equal(y_auto.view(np.uint16), y_gemm.view(np.uint16))
-    assert same_gemv or same_gemm
+    forced = {v: run_layer(L, x, v) for v in (2, 5, GEMM)}      # tensor-core GEMV, table-driven GEMV, GEMM
+    same = {v: np.array_equal(y_auto.view(np.uint16), y.view(np.uint16)) for v, y in forced.items()}
+    assert any(same.values())
     if batch <= 4:
-        assert same_gemv
+        assert same[2] or same[5]
     if batch == 16:
-        assert same_gemm
+        assert same[GEMM]
 
 
 DEQ = 4     # variant number of the GEMM on dequantised fp16 weight tiles
@@ -114,7 +113,7 @@ def test_dequantised_tile_gemm(K, M, N, batch):
     L = make_layer(M, N, K, key=(64, K, M, N))
     x = make_x(batch, N, key=(64, M, N, batch))
     y = run_layer(L, x, DEQ)
-    err, tol = check_against_oracle(L, x, y)
+    err, tol = check_against_oracle(L, x, y, tight=False)          # fp16-rounded weights: the mandated bound only
     y_exact = run_layer(L, x, GEMM)
     err_exact, _ = check_against_oracle(L, x, y_exact)
     assert err_exact.max() <= err.max() + 1e-3 * tol.max()        # the exact expansion is never noticeably worse
@@ -138,12 +137,12 @@ def test_gemm_split_contraction_across_a_cluster(K, M, N, batch, variant):
     x = make_x(batch, N, key=(65, M, N, batch))
     y = run_layer(L, x, variant)
     if M * N * batch <= 2 ** 31:
-        check_against_oracle(L, x, y)
-    else:                                           # large case: sampled rows
-        rows = np.unique(np.concatenate([np.arange(0, 4), np.arange(126, 131), np.arange(M - 3, M), np.random.default_rng(0).integers(0, M, 24)]))
-        from oracle import rabit_oracle as orc
-        ref = orc.linear(L.planes[:, rows, :], L.g[:, rows], L.h, x)
-        tol = orc.tolerance(L.g, L.h, x)
-        assert (np.abs(y[:, rows].astype(np.float64) - ref).max(axis=1) <= tol).all()
+        check_against_oracle(L, x, y, tight=variant != DEQ)
+    else:                                           # large case: sampled rows, at least one in every 128-row tile
+        rng = np.random.default_rng(0)
+        rows = np.unique(np.concatenate([np.arange(0, 4), np.arange(126, 131), np.arange(M - 3, M), rng.integers(0, M, 24),
+                                         np.arange(0, M, 128) + rng.integers(0, 128, (M + 127) // 128)]))
+        rows = rows[rows < M]
+        check_against_oracle(L, x, y, tight=variant != DEQ, rows=rows)
     y2 = run_layer(L, x, variant)
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
