@@ -13,6 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librabit.so")
 LIB_TRACE = os.path.join(HERE, "librabit_trace.so")          # the same sources with -DRABIT_TRACE (phase stamps)
+LIB_CHECKED = os.path.join(HERE, "librabit_checked.so")      # the same sources with -DRABIT_CHECKED (index checks in the decode kernel)
 SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemv_lut.cu", "rabit_gemm_tc.cu",
            "rabit_noalloc.cu", "rabit_derive.cu", "rabit_selftest.cu"]
 NVCC_FLAGS = [
@@ -34,12 +35,12 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
-    if not trace and not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, trace: bool = False, checked: bool = False) -> str:
+    if not trace and not checked and not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    out = LIB_TRACE if trace else LIB
-    cmd = [nvcc] + NVCC_FLAGS + (["-DRABIT_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else []) + ["-o", out] + _sources()
+    out = LIB_TRACE if trace else LIB_CHECKED if checked else LIB
+    cmd = [nvcc] + NVCC_FLAGS + (["-DRABIT_TRACE"] if trace else []) + (["-DRABIT_CHECKED"] if checked else []) + (["-Xptxas", "-v"] if verbose else []) + ["-o", out] + _sources()
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode != 0:
         sys.stderr.write(proc.stdout + proc.stderr)
@@ -49,4 +50,4 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, trace="--trace" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, trace="--trace" in sys.argv, checked="--checked" in sys.argv))

@@ -88,6 +88,7 @@ struct CtaRange {
 };
 struct LutParams {
     int n_layers;
+    unsigned int* status;           // RABIT_CHECKED builds: set to 2 when an index check fails (the access is skipped)
     unsigned long long* trace;      // RABIT_TRACE builds: 8 time stamps per CTA of this launch (nullptr: none)
     LutLayer layer[kMaxGroup];
     CtaRange range[kMaxGrid];
@@ -153,6 +154,16 @@ __device__ __forceinline__ unsigned long long sm_clock() {
 #define RABIT_STAMP(i) do { } while (0)
 #endif
 
+// Checked build (-DRABIT_CHECKED, python paper_2602_05367_b200/build.py --checked): every index that addresses global or
+// shared memory in this kernel is compared with its range first; a violation sets the status word to 2 and the access
+// is skipped (never a trap, never an out-of-range access), so the small-shape suite can run under it in place of a
+// memory checker.
+#ifdef RABIT_CHECKED
+#define RABIT_IN_RANGE(cond) ((cond) ? true : (atomicExch(P.status, 2u), false))
+#else
+#define RABIT_IN_RANGE(cond) true
+#endif
+
 template <int K>
 struct Blk {
     uint4 v[2 * K];                  // one lane's 32 bytes per path: (path k, half hf) at v[2k + hf]
@@ -186,7 +197,7 @@ __device__ __forceinline__ void settle(Pending (&pd)[NB], const LutLayer& L) {
         const bool poisoned = pd[b].bad || (pd[b].old >> 63) != 0;
         const float v = poisoned ? __int_as_float(0x7FC00000) : __ll2float_rn(total) * L.unit;
         const long long row = (pd[b].word - L.acc) - (long long)b * L.Mp;       // (rare path: the layer's fields come from shared memory)
-        if (row < L.M) L.y[(size_t)b * L.M + row] = __float2half_rn(v);
+        if (row >= 0 && row < L.M) L.y[(size_t)b * L.M + row] = __float2half_rn(v);
         *pd[b].word = 0ULL;                                                     // resting state for the next call
     }
 }
@@ -290,7 +301,9 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
                 }
                 const uint32_t dst = tab0 + b * T::kBytes + (k >> 1) * 65536 + (ehi * 32) * 256 + (k & 1) * 128 + lane * 4;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) sts_f32(dst + e * 256, v[e]);
+                for (int e = 0; e < 32; ++e)
+                    if (RABIT_IN_RANGE(dst + e * 256 >= tab0 && dst + e * 256 + 4 <= tab0 + (uint32_t)(NB * T::kBytes) && dst + e * 256 + 4 <= smem_u32(smem) + (uint32_t)T::kSmem))
+                        sts_f32(dst + e * 256, v[e]);
             }
         }
     };
@@ -345,11 +358,18 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
         const int row = (seg_rb0 + (bb - seg_begin)) * RABIT_LUT_ROWS + lane;
         unsigned short graw[K];
 #pragma unroll
-        for (int k = 0; k < K; ++k) graw[k] = ldg_u16_early(g_base + (size_t)k * Mp + row);
-        Blk<K> nxt = load_blk<K>(range_base, i + 1 < n_mine ? bb + kWarps : bb, lane);   // (the last iteration re-reads its own block: in bounds, unused)
+        for (int k = 0; k < K; ++k) {
+            graw[k] = 0;
+            if (RABIT_IN_RANGE(row >= 0 && row < Mp)) graw[k] = ldg_u16_early(g_base + (size_t)k * Mp + row);
+        }
+        const int bb_next = i + 1 < n_mine ? bb + kWarps : bb;
+        Blk<K> nxt = cur;
+        if (RABIT_IN_RANGE(bb_next >= 0 && bb_next < n_blocks && (long long)R.b0 + bb_next < (long long)L.n_cs * L.n_rb))
+            nxt = load_blk<K>(range_base, bb_next, lane);   // (the last iteration re-reads its own block: in bounds, unused)
         if (owe) {
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
+                if (!RABIT_IN_RANGE(pd[b].word >= acc_base && pd[b].word < acc_base + (size_t)NB * Mp)) continue;
                 if (pd[b].bad) atomicOr(pd[b].word, 1ULL << 63);
                 pd[b].old = atomicAdd(pd[b].word, pd[b].add);
                 pd[b].live = true;
@@ -380,6 +400,12 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
                 // address = table base | sign byte << 8 | bank offset, all from one permute
                 const uint32_t a0 = prmt(w, c[j][0], 0x7604), a1 = prmt(w, c[j][0], 0x7615);
                 const uint32_t a2 = prmt(w, c[j][1], 0x7624), a3 = prmt(w, c[j][1], 0x7635);
+#ifdef RABIT_CHECKED
+                {
+                    const uint32_t lo = tab0, hi = tab0 + 65536u - 128u;     // with the path offset added: inside table k >> 1
+                    if (!RABIT_IN_RANGE(a0 >= lo && a0 < hi && a1 >= lo && a1 < hi && a2 >= lo && a2 < hi && a3 >= lo && a3 < hi)) return;
+                }
+#endif
                 static_for<0, NB>([&](auto bc) {
                     constexpr int b = decltype(bc)::value;
                     acc[b][k][0] += lds_f32<T::offset(k, b)>(a0);
@@ -423,6 +449,7 @@ rabit_gemv_lut_kernel(const __grid_constant__ LutParams P) {
     if (owe) {
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
+            if (!RABIT_IN_RANGE(pd[b].word >= acc_base && pd[b].word < acc_base + (size_t)NB * Mp)) continue;
             if (pd[b].bad) atomicOr(pd[b].word, 1ULL << 63);
             pd[b].old = atomicAdd(pd[b].word, pd[b].add);
             pd[b].live = true;
@@ -441,7 +468,9 @@ struct Cost {
 };
 // SM clock cycles, from the phase stamps of the kernel on B200: a block of K paths (look-ups, loads, its atomic) and a
 // table (build plus the two barriers around it).
-Cost cost_of(int K, int nb) { return Cost{(long long)nb * (70 * K + 30), (long long)nb * (200 * K) + 100}; }
+// (the table figure is a fit: the split that minimises the measured step time charges a table about 26 blocks, far
+// more than its 430 cycles of stores, because a rebuild in mid-range also stops every warp at two barriers)
+Cost cost_of(int K, int nb) { return Cost{(long long)nb * (70 * K + 30), (long long)nb * (2200 * K) + 100}; }
 
 // CTAs a layer of n_cs x n_rb blocks needs when no CTA may cost more than `limit`; writes the cuts if asked.
 int ctas_needed(int n_cs, int n_rb, const Cost& C, long long limit, std::vector<int>* cuts) {
@@ -536,7 +565,7 @@ cudaError_t rabit_launch_gemv_lut_group(const rabit_layer* const* layers, int n_
     const int K = layers[0]->geom.K;
     LutParams P;
     P.n_layers = n_layers;
-    (void)status_override;                                               // this kernel has no wait that could run out
+    P.status = status_override ? status_override : layers[0]->d_status;  // (only a checked build writes it: this kernel has no wait that could run out)
     P.trace = nullptr;
     const Cost C = cost_of(K, batch);
     long long weight[kMaxGroup], total_weight = 0, total_blocks = 0;

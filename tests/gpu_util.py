@@ -16,6 +16,7 @@ def run_layer(layer_inputs, x_np, variant=0, device="cuda:0"):
         x = torch.from_numpy(np.ascontiguousarray(x_np)).to(device)
         y = rabit.rabit_linear(L, x)
         torch.cuda.synchronize()
+        assert L.status() == 0, rabit.last_error()          # no bounded wait ran out, no index check of a checked build failed
         return y.cpu().numpy()
     finally:
         L.free()
