@@ -46,12 +46,13 @@ typedef enum rabit_status {
 
 typedef struct rabit_layer rabit_layer;   /* opaque host-side descriptor */
 
-/* Version of the packed device layout written by rabit_pack_host (also stored in its header). */
+/* Version of the packed device layout written by rabit_pack_host (also stored in its header): 3. */
 RABIT_API int rabit_layout_version(void);
 
 /*
- * Bytes of the packed image of a K x M x N layer: header + interleaved sign tiles + padded
- * fp16 scales + the per-layer reduction scratch.  Returns 0 for an unsupported shape.
+ * Bytes of the packed image of a K x M x N layer: header + the sign bits in two arrangements (tiles for the
+ * tensor-core kernels, byte look-up blocks for the table-driven decode kernel: 2K bits per weight in device memory,
+ * of which a call reads K) + padded fp16 scales + the per-layer reduction scratch.  Returns 0 for an unsupported shape.
  * (Storage accounting of Section 4.1: K bits per weight plus the scale vectors.)
  */
 RABIT_API size_t rabit_packed_bytes(int K, int M, int N);
@@ -113,10 +114,13 @@ RABIT_API int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uin
  *   x  DEVICE fp16 [batch][N] row-major, 16-byte aligned
  *   y  DEVICE fp16 [batch][M] row-major, 16-byte aligned, must not overlap x
  * Asynchronous on `stream`; allocates nothing, never synchronises, and may be captured in
- * a CUDA graph.  Up to 4 batch rows run the bandwidth-bound GEMV (one pass over the weights), more
- * than 16 the tensor-core GEMM; in between, GEMV passes of four rows or one GEMM launch, whichever the
- * library's cost estimate for this shape favours.  A GEMM with few output tiles runs as clusters of CTAs
- * that share a tile's contraction.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end.
+ * a CUDA graph.  The layer's device must be the current device.  One or two batch rows run the table-driven
+ * GEMV (one pass over the weights: a shared-memory table of the partial sums of h*x over eight columns, indexed by the
+ * packed sign byte; also three or four rows on layers up to 8 MB, as two passes), three or four rows otherwise the
+ * integer tensor-core GEMV (one pass), more than 16 the tcgen05 GEMM; in between, tensor-core GEMV passes of four rows or
+ * one GEMM launch, whichever the library's cost estimate for this shape favours.  A GEMM with few output tiles runs as
+ * clusters of CTAs that share a tile's contraction.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end;
+ * an inf or NaN in a batch row of x makes that row of y non-finite and leaves the other rows untouched.
  */
 RABIT_API int rabit_linear(const rabit_layer* layer, const void* x, void* y, int batch, void* stream);
 
@@ -259,7 +263,8 @@ RABIT_API int rabit_layer_N(const rabit_layer* layer);
  *   0 = automatic (default), 1 = plain sign-select kernel, 2 = integer tensor-core GEMV,
  *   3 = tcgen05 GEMM with one exact +-h_k operand tile and accumulator per path,
  *   4 = tcgen05 GEMM on the dequantised weight tile sum_k +-g_k h_k rounded to fp16 (Eq. 2 formed per tile; one
- *       contraction of length N instead of K of them; never chosen automatically: it rounds every weight to fp16).
+ *       contraction of length N instead of K of them; never chosen automatically: it rounds every weight to fp16),
+ *   5 = table-driven GEMV (passes of up to two batch rows; N up to 65280).
  * Returns RABIT_INVALID_ARG for a variant that cannot run the layer.
  * Meant for A/B timing and profiling; results are within tolerance for every variant.
  */

@@ -51,6 +51,28 @@ def test_derived_planes_bit_exact_and_layer_parity(K, M, N):
     layer.free()
 
 
+def test_derive_then_run_on_one_stream_without_a_sync():
+    """The decode kernel starts reading weights before its dependency wait; a layer derived on the same stream just
+    before must still be seen complete (the library orders the two with a fill after the derivation kernels)."""
+    import torch
+    import paper_2602_05367_b200 as rabit
+    K, M, N = 2, 4096, 4096
+    W, g, h = _inputs(K, M, N, seed=77)
+    Wd = torch.from_numpy(W).cuda()
+    x = make_x(1, N, key=(91, N))
+    xd = torch.from_numpy(x).cuda()
+    torch.cuda.synchronize()
+    for rep in range(3):
+        layer = rabit.rabit_derive_pack(Wd, g, h)                         # asynchronous
+        y = rabit.rabit_linear(layer, xd)                                 # same stream, nothing in between
+        torch.cuda.synchronize()
+        class L:
+            pass
+        L.planes, L.g, L.h = orc.derive_planes(W, g, h, dtype=np.float32), g, h
+        check_against_oracle(L, x, y.cpu().numpy())
+        layer.free()
+
+
 def test_derive_pack_argument_errors():
     import ctypes
     import torch

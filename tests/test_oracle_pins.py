@@ -308,3 +308,30 @@ def test_generator_recipe():
     assert np.array_equal(L.planes, L2.planes) and np.array_equal(L.g, L2.g)
     L3 = make_layer(256, 512, 2, key=(0, 0, 1))
     assert not np.array_equal(L.planes, L3.planes)
+
+
+def _derive_inputs(K, M, N, seed):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((M, N)) * 0.02).astype(np.float32)
+    h = rng.uniform(0.5, 1.5, (K, N)).astype(np.float16)
+    g = np.empty((K, M), dtype=np.float16)
+    scale = 0.016
+    for k in range(K):
+        g[k] = (scale * rng.uniform(0.8, 1.2, M)).astype(np.float16)
+        scale *= 0.45
+    return W, g, h
+
+
+def test_float32_and_float64_readings_differ_only_at_near_ties():
+    """Reading R13: the device keeps the residual in fp32.  Against the float64 recurrence of the oracle the planes may
+    differ only where a residual is within rounding distance of zero; counted and bounded here."""
+    W, g, h = _derive_inputs(3, 512, 1024, seed=5)
+    p32 = orc.derive_planes(W, g, h, dtype=np.float32)
+    p64 = orc.derive_planes(W, g, h, dtype=np.float64)
+    diff = np.unpackbits((p32 ^ p64).view(np.uint8)).sum()
+    total = p32.size * 32
+    assert np.array_equal(p32[0], p64[0])                                 # the first plane is sign(W) in both
+    assert diff / total < 1e-5, f"{diff} of {total} signs differ"
+    print(f"fp32 vs float64 derivation: {diff} of {total} signs differ ({diff / total:.2e})")
+
+
