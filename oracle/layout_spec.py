@@ -6,7 +6,7 @@ library image can be compared byte for byte.  The paper fixes only the sign -> b
 
 Image = header (256 B) | sign tiles | g fp16 [K][Mp] | h fp16 [K][N] | fp32 partial scratch
 [n_rt*K + max_grid][partial_batch][128] | u32 flags [n_rt*K + max_grid] + one status word |
-look-up blocks | u64 accumulate words [4][Mp]; every section starts on a 256-byte boundary;
+look-up blocks | u64 accumulate words [16][Mp]; every section starts on a 256-byte boundary;
 padding, flags (reserved), status and accumulate words are zero, the partial scratch section is
 filled with 0xFF bytes (its resting state: "nothing written yet").
 Mp = M rounded up to 128; padded signs are +1 (bit 0), padded scales 0; N is a multiple of
@@ -49,7 +49,7 @@ PARTIAL_BATCH = 4
 LUT_ROWS = 32
 LUT_COLS = 256
 LUT_PART_BYTES = 1024
-LUT_MAX_BATCH = 4
+LUT_MAX_BATCH = 16
 _HEADER_FMT = "<14I2IIi2I8Q"
 _HEADER_KEYS = ["magic", "version", "K", "M", "N", "Mp", "n_rt", "n_ct", "max_grid", "partial_batch",
                 "hmax0", "hmax1", "hmax2", "hmax3", "n_rb", "n_cs", "fix_bits", "unit_exp", "reserved0", "reserved1",

@@ -166,17 +166,18 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
         const double packed_mb = (double)G.K * G.Mp * G.N / 8.0e6;
         if (rabit_gemv_lut_supports(*layer, batch)) {
             variant = 5;
+        } else if (rabit_gemv_f16_supports(*layer, batch)) {
+            variant = 6;                    // 3..16 rows: one pass over the weights with the batch in the MMA's N dimension
         } else if (batch <= 4 && packed_mb <= 8.0 && rabit_gemv_lut_supports(*layer, 1)) {
-            variant = 5;                    // two passes of the table-driven kernel: measured faster than one pass of the tensor-core GEMV on small layers
+            variant = 5;                    // two passes of the table-driven kernel
         } else if (batch <= RABIT_MAX_GEMV_BATCH) {
             variant = rabit_gemv_mma_supports(*layer, batch) ? 2 : 1;
-            // From 5 batch rows on the GEMV makes two to four passes over the weights; the tensor-core GEMM, whose cost
-            // does not depend on the batch up to 256, is then often cheaper.  Both estimates are fits to measurements
-            // on B200 (us): a GEMV pass of four rows costs 10 + max(0, packed MB - 4) / 1.3.
+            // From 5 batch rows on the integer-MMA GEMV makes two to four passes over the weights; the tensor-core GEMM,
+            // whose cost does not depend on the batch up to 256, is then often cheaper.  Both estimates are fits to
+            // measurements on B200 (us): a GEMV pass of four rows costs 10 + max(0, packed MB - 4) / 1.3.
             if (variant == 2 && batch > 4 && rabit_gemm_tc_supports(*layer, batch)) {
                 const double passes = (double)((batch + rabit_gemv_mma_max_rows() - 1) / rabit_gemv_mma_max_rows());
-                const double mb = (double)G.K * G.Mp * G.N / 8.0e6;
-                const double gemv_us = passes * (10.0 + (mb > 4.0 ? (mb - 4.0) / 1.3 : 0.0));
+                const double gemv_us = passes * (10.0 + (packed_mb > 4.0 ? (packed_mb - 4.0) / 1.3 : 0.0));
                 const double gemm_us = rabit_gemm_tc_estimate_us(*layer, batch);
                 if (gemm_us < 0.9 * gemv_us) variant = 3;
             }
@@ -214,6 +215,11 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
                                           batch - b0 >= rows ? rows : batch - b0, st);
             break;
         }
+        case 6:
+            if (!rabit_gemv_f16_supports(*layer, batch))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: f16 tensor-core GEMV cannot run batch %d", batch);
+            e = rabit_launch_gemv_f16(*layer, x, y, batch, st);
+            break;
         default:
             e = rabit_launch_plain(*layer, x, y, batch, st);
             break;
@@ -257,6 +263,17 @@ extern "C" int rabit_linear_group(const rabit_layer* const* layers, const void* 
         if (lut) {
             cudaError_t e = rabit_launch_gemv_lut_group(layers, n_layers, xs, ys, batch, st, nullptr, nullptr);
             if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_linear_group: launch failed: %s", cudaGetErrorString(e));
+            return RABIT_OK;
+        }
+    }
+    {
+        bool f16 = true;                                         // 3..16 rows: every layer takes the f16 tensor-core GEMV, launch by launch
+        for (int l = 0; l < n_layers && f16; ++l) f16 = layers[l]->variant == 0 && rabit_gemv_f16_supports(*layers[l], batch);
+        if (f16) {
+            for (int l = 0; l < n_layers; ++l) {
+                int rc = rabit_linear(layers[l], xs[l], ys[l], batch, stream);
+                if (rc != RABIT_OK) return rc;
+            }
             return RABIT_OK;
         }
     }
@@ -486,7 +503,7 @@ extern "C" int rabit_layer_N(const rabit_layer* layer) { return layer ? layer->g
 extern "C" int rabit_set_variant(rabit_layer* layer, int variant) {
     rabit_clear_error();
     if (!layer) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: layer is NULL");
-    if (variant < 0 || variant > 5) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..5");
+    if (variant < 0 || variant > 6) return rabit_fail(RABIT_INVALID_ARG, "rabit_set_variant: variant must be 0..6");
     layer->variant = variant;
     return RABIT_OK;
 }

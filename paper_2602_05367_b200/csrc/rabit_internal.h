@@ -12,7 +12,7 @@
 struct rabit_layer {
     RabitGeom geom;
     int device;
-    int variant;                 // 0 auto, 1 plain, 2 integer-MMA GEMV, 3 tcgen05 GEMM, 4 dequantised-tile GEMM, 5 table-driven GEMV
+    int variant;                 // 0 auto, 1 plain, 2 integer-MMA GEMV, 3 tcgen05 GEMM, 4 dequantised-tile GEMM, 5 table-driven GEMV, 6 f16 tensor-core GEMV
     int sm_count;
     char* dev_base;              // caller-owned packed image
     size_t dev_bytes;
@@ -67,6 +67,10 @@ unsigned int* rabit_static_scratch_status(int device);   // rabit_noalloc.cu; nu
 // Phase tracing (rabit_api.cu): the next free record of 8 stamps x `ctas` in the caller's trace buffer, or nullptr
 // when tracing is off, the buffer is full or the library was built without RABIT_TRACE.
 unsigned long long* rabit_trace_slot(int ctas);
+
+// f16 tensor-core GEMV for 3..16 batch rows (rabit_gemv_f16.cu)
+cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
+bool rabit_gemv_f16_supports(const rabit_layer& L, int batch);
 
 // table-driven GEMV (rabit_gemv_lut.cu); acc_override / status_override redirect the scratch (nullptr: the image's own)
 cudaError_t rabit_launch_gemv_lut(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);

@@ -6,7 +6,7 @@
 //   header | sign tiles | g fp16 [K][Mp] | h fp16 [K][N] | fp32 partial scratch | flags + status |
 //   look-up blocks | u64 accumulate words
 //
-// (1) Sign tiles (tensor-core kernels: the integer-MMA GEMV of batches 3..16 and the tcgen05 GEMM).
+// (1) Sign tiles (tensor-core kernels: the f16 and integer-MMA GEMVs of batches 3..16 and the tcgen05 GEMM).
 // The sign bits of each path are cut into tiles of 128 output rows x 32 input columns.
 // One tile is 512 bytes = 32 lanes x 16 bytes, so a warp reads a tile with one 128-bit
 // access per lane.  The eight bits of every byte belong to eight different 16-row blocks of
@@ -66,7 +66,7 @@
 #define RABIT_LUT_ROWS 32       /* output rows of a look-up block (one per lane) */
 #define RABIT_LUT_COLS 256      /* input columns of a slice (32 byte groups) */
 #define RABIT_LUT_PART_BYTES 1024   /* one path of one block */
-#define RABIT_LUT_MAX_BATCH 4   /* batch rows the accumulate words provide for */
+#define RABIT_LUT_MAX_BATCH 16  /* batch rows the accumulate words provide for */
 #define RABIT_LUT_MAX_SLICES 255    /* the arrival count of an accumulate word has eight bits */
 
 struct RabitHeader {            // first 256 bytes of a packed image (little endian)

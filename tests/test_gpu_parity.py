@@ -12,7 +12,7 @@ from tests.gpu_util import run_layer, check_against_oracle
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [0, 1, 2, 5]   # automatic, plain sign-select, integer-MMA GEMV, table-driven GEMV
+VARIANTS = [0, 1, 2, 5, 6]   # automatic, plain sign-select, integer-MMA GEMV, table-driven GEMV, f16 tensor-core GEMV
 
 SMALL = [  # several tiles plus ragged tails in both dimensions
     (2, 32, 128), (2, 100, 160), (2, 256, 1184), (3, 96, 640), (1, 33, 96), (2, 160, 2080), (2, 1000, 512),
@@ -37,6 +37,18 @@ def test_batches(batch, variant):
     x = make_x(batch, 896, key=(71, batch))
     y = run_layer(L, x, variant)
     check_against_oracle(L, x, y)
+
+
+@pytest.mark.parametrize("K,M,N", [(2, 192, 896), (3, 300, 640), (1, 129, 288), (2, 1000, 4352), (2, 4096, 4096)])
+@pytest.mark.parametrize("batch", [3, 7, 8, 9, 16])
+def test_f16_tensor_core_gemv_batches(K, M, N, batch):
+    """The batch 3..16 kernel (batch in the MMA's N dimension) forced, every batch width class, ragged shapes, K = 1..3."""
+    L = make_layer(M, N, K, key=(69, K, M, N))
+    x = make_x(batch, N, key=(69, M, N, batch))
+    y = run_layer(L, x, 6)
+    check_against_oracle(L, x, y)
+    y2 = run_layer(L, x, 6)
+    assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))     # integer accumulate words: the same bits every run
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
