@@ -6,26 +6,38 @@
 // eight columns per batch row and needs a pass over x first.  Here the A operand of mma.sync.m16n8k16 is +-h_k expanded in
 // registers from the sign tiles (the weight bit flips the sign bit of the fp16 input scale: exact), B is x as it is, the
 // accumulators are fp32: products are exact, 8 batch rows per MMA and 16 with a second MMA on the same A, no digits, no
-// scale search.  The cost is that of the expansion (five logic instructions per two A registers) and does not depend on
-// the batch.
+// scale search.  The cost is that of the expansion and does not depend on the batch.
+//
+// Expansion.  Shifts, byte permutes and logic instructions all issue on the half-rate integer pipe of an SM sub-partition
+// (16 lanes per clock), and that pipe, not the tensor pipe, bounds this kernel.  So an A register (two fp16 values) costs
+// ONE logic instruction there, (v & 0x80008000) ^ h, and the shift that brings the two weight bits to bits 15 and 31 is a
+// multiplication by a power of two on the multiply-add pipe: v = w * 2^s, where the factor comes from a kernel parameter
+// so that the compiler keeps it a multiplication.  The two bits must be 16 apart in the word, i.e. two columns apart:
 //
 // Operand mapping.  A sign tile (rabit_layout.h) gives lane (gq, tq) four words w[a]; byte c of word a has in bit p the
 // sign of row 16p + gq + 8(a & 1), column 16(a >> 1) + 4tq + c of the tile.  For the k-step kh = a >> 1 (16 columns) and
 // the row block p, the MMA's k slots (2tq, 2tq+1, 2tq+8, 2tq+9) of lane (gq, tq) are taken to be the tile columns
-// 16kh + 4tq + (0, 1, 2, 3): any fixed assignment of slots to columns is valid as long as A and B use the same one.  Then
-//     a0 = +-h(cols 0,1) for row gq      from bytes 0,1 of w[2kh]         a1 = the same columns, row gq + 8, from w[2kh+1]
-//     a2 = +-h(cols 2,3) for row gq      from bytes 2,3 of w[2kh]         a3 = row gq + 8, from w[2kh+1]
-//     b0 = x[n = gq][cols 0,1]           b1 = x[n = gq][cols 2,3]         (one 8-byte load per lane and k-step)
+// 16kh + 4tq + (0, 2, 1, 3): any fixed assignment of slots to columns is valid as long as A and B use the same one.  Then
+//     a0 = +-h(cols 0,2) for row gq      from bits p, 16+p of w[2kh] * 2^(15-p)      a1 = the same, row gq + 8, from w[2kh+1]
+//     a2 = +-h(cols 1,3) for row gq      from bits 8+p, 24+p of w[2kh] * 2^(7-p)     a3 = row gq + 8, from w[2kh+1]
+//     b0 = x[n = gq][cols 0,2]           b1 = x[n = gq][cols 1,3]         (one 8-byte load per lane and k-step, two permutes)
 // and the accumulator lane holds rows gq, gq + 8 of the block and batch rows 2tq, 2tq + 1.
 //
-// Work split.  A unit is (row tile of 128 rows) x (a range of whole 256-column slices), all paths.  One CTA of 8 warps per
-// unit; warp w works on path w % K and shares the column tiles of the range with the other warps of that path, one
-// 512-byte tile per 128-bit load per lane, several tiles ahead.  At the end every warp scales its accumulators by g_k and
-// writes them to its own slot of shared memory, the CTA adds the slots in a fixed order (deterministic), and every output
-// of the unit goes, as in the table-driven kernel, into the row's 64-bit accumulate word with one integer atomic
-// (fixed-point grid of the packer, arrival count in bits 55..62, bit 63 = non-finite); the lane whose add completes a row
-// rounds it to fp16, stores y and clears the word.  A contribution that covers s slices is shifted by s * 2^fix_bits, so
-// the total shift is the same n_cs * 2^fix_bits for every split.  Nothing waits for another CTA.
+// Work split.  The layer is n_rt row tiles x n_cs slices of 256 columns; in that order the (row tile, slice) pairs are cut
+// into one contiguous range per CTA, all the same length to within one pair.  The part of a range inside one row tile is a
+// segment.  CTAs of 8 warps, two per SM (while one adds up a segment and waits for its atomics the other computes; one
+// CTA of 16 warps per SM measured 15 % slower); warp w works on path w % K and shares the column tiles of the segment with the other warps
+// of that path.  A warp streams its tiles through a ring of its own in shared memory with asynchronous 16-byte copies
+// (one per lane and tile, each lane reads back only what it copied itself, so no barrier is involved), kRing - 1 tiles
+// ahead: with 16 warps per SM that keeps about 56 KB per SM in flight, which is what the HBM latency needs (with the
+// tiles prefetched into registers, two to four per warp, the kernel ran at the speed of its memory latency, 1.1 to
+// 1.7 TB/s).  At the end of a segment every warp writes
+// its accumulators to its own slot of shared memory, the CTA adds the slots path by path in a fixed order (deterministic)
+// and applies g_k to each path's sum, and every output of the segment goes, as in the table-driven kernel, into the row's 64-bit accumulate
+// word with one integer atomic (fixed-point grid of the packer, arrival count in bits 55..62, bit 63 = non-finite); the
+// lane whose add completes a row (the count reaches the number of segments of that row tile) rounds it to fp16, stores y
+// and clears the word.  A contribution that covers s slices is shifted by s * 2^fix_bits, so the total shift is the same
+// n_cs * 2^fix_bits for every split.  Nothing waits for another CTA.
 #include <cuda_fp16.h>
 
 #include <algorithm>
@@ -37,7 +49,8 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kMaxUnits = 1 << 20;
+constexpr int kRing = 8;                               // sign tiles a warp keeps in flight or in use (a power of two)
+constexpr long long kMaxPairs = 1LL << 30;
 constexpr unsigned long long kSumMask = (1ULL << 55) - 1;
 
 struct F16Params {
@@ -49,10 +62,10 @@ struct F16Params {
     unsigned long long* acc;        // [16][Mp], all zero between calls
     int K, M, N, Mp, n_rt, n_ct, n_cs;
     int batch;
-    int splits;                     // column ranges per row tile; range r covers slices [r * n_cs / splits, (r + 1) * n_cs / splits)
-    int n_units;                    // n_rt * splits
+    int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; CTA c owns pairs [c * n_pairs / grid, (c + 1) * n_pairs / grid)
     int fix_bits;
     float inv_unit, unit, limit;
+    uint32_t two, two_pow_8;        // 2 and 256: multipliers the compiler cannot fold into shifts
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
@@ -63,7 +76,13 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
 // (a & 0x80008000) ^ c: the sign bits of two fp16 values, applied to a pair of input scales
 __device__ __forceinline__ uint32_t flip(uint32_t a, uint32_t c) {
     uint32_t r;
-    asm("lop3.b32 %0, %1, 0x80008000, %2, 0x6A;" : "=r"(r) : "r"(a), "r"(c));
+    asm volatile("lop3.b32 %0, %1, 0x80008000, %2, 0x6A;" : "=r"(r) : "r"(a), "r"(c));
+    return r;
+}
+// a * m on the multiply-add pipe (m is a power of two the compiler does not know)
+__device__ __forceinline__ uint32_t mul_lo(uint32_t a, uint32_t m) {
+    uint32_t r;
+    asm volatile("mul.lo.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(m));
     return r;
 }
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -71,39 +90,98 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+// 16 bytes global -> shared, asynchronous, not through L1; one group per call so that groups and tiles count alike
+__device__ __forceinline__ void copy_async_16(uint32_t dst_smem, const void* src, bool valid) {
+    if (valid) asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void copy_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds_128(uint32_t addr) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::128B.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
 
-// What a warp needs besides the sign words for one column tile of its path.
-template <int NH>
-struct Feed {
-    uint2 h[2];                      // input scales of its four columns, per k-step
-    uint2 x[2][NH];                  // activations of its four columns, per k-step and half of the batch
-};
+// One output of a segment from the warps' slots: warp w holds path w % KK; the paths' sums are formed warp by warp in the
+// order of the warps and scaled by the path's output scale.
+template <int KK, int NH>
+__device__ __forceinline__ float path_sums(const float* col, const __half (&g)[RABIT_MAX_K]) {
+    float sk[KK];
+#pragma unroll
+    for (int kk = 0; kk < KK; ++kk) sk[kk] = 0.f;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) sk[wv % KK] += col[(size_t)wv * (NH * 8 * 128)];
+    float v = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < KK; ++kk) v = fmaf(__half2float(g[kk]), sk[kk], v);
+    return v;
+}
 
-// NH = halves of the batch (8 rows each) a pass carries; DEPTH = sign tiles a warp keeps in flight.
-template <int NH, int DEPTH>
+// First CTA whose range holds pair u:  the largest c with  c * n_pairs / grid <= u.
+__device__ __forceinline__ int owner_of(long long u, int n_pairs, int grid) {
+    return (int)(((u + 1) * grid - 1) / n_pairs);
+}
+
+// NH = halves of the batch (8 rows each) a pass carries.
+template <int NH>
 __global__ void __launch_bounds__(kThreads, 2)
 rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
-    extern __shared__ __align__(16) float slots[];                       // [kWarps][NH * 8][128] scaled partial outputs
+    extern __shared__ __align__(16) float slots[];                       // [kWarps][NH * 8][128] scaled partial outputs, then the rings
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tq = lane & 3;
+    // the lane's 16 bytes of ring slot 0 of its warp; slot r is r * 512 bytes further
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(slots) + (uint32_t)(kWarps * NH * 8 * 128 * sizeof(float)) +
+                          (uint32_t)((warp * kRing * 32 + lane) * 16);
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool waited = false;
 
-    for (int unit = blockIdx.x; unit < P.n_units; unit += gridDim.x) {
-        const int rt = unit / P.splits, r = unit - rt * P.splits;
-        const int s0 = (int)((long long)r * P.n_cs / P.splits), s1 = (int)((long long)(r + 1) * P.n_cs / P.splits);
-        const int c0 = s0 * 8, c1 = min(P.n_ct, s1 * 8);                 // column tiles of the range (a slice is eight of them)
-        // every warp works on ONE path: path k = warp % K, and the column tiles of the range are dealt out among the warps of
-        // that path (K = 3: three, three and two warps)
-        const int k = warp % P.K;
-        const int n_same = (kWarps - k + P.K - 1) / P.K, j0 = warp / P.K;
+    // every warp works on ONE path: path k = warp % K, and the column tiles of a segment are dealt out among the warps of
+    // that path (K = 3: three, three and two warps)
+    const int k = warp % P.K;
+    const int n_same = (kWarps - k + P.K - 1) / P.K, j0 = warp / P.K;
+    const int hk = k * P.N + 4 * tq;                                      // element offsets (K * N and 16 * N fit 31 bits: N <= 65280)
+    int xb[NH];
+#pragma unroll
+    for (int hf = 0; hf < NH; ++hf)                                      // lanes beyond the batch read its last row; their columns are never stored
+        xb[hf] = min(8 * hf + gq, P.batch - 1) * P.N + 4 * tq;
 
+    // A segment: row tile rt, column tiles [ct0, c1) of which this warp takes every n_same-th, starting at ct0.
+    struct Segment {
+        int rt, n_slices, c1, ct0, n_my;
+        const uint4* wsrc;                                               // the warp's first tile (this lane's 16 bytes)
+    };
+    long long u = (long long)blockIdx.x * P.n_pairs / gridDim.x;
+    const long long u_end = (long long)(blockIdx.x + 1) * P.n_pairs / gridDim.x;
+    auto next_segment = [&]() {                                          // the segment that starts at pair u; advances u
+        Segment sg;
+        sg.rt = (int)(u / P.n_cs);
+        const int s0 = (int)(u - (long long)sg.rt * P.n_cs);
+        const int s1 = (int)min((long long)P.n_cs, s0 + (u_end - u));
+        u += s1 - s0;
+        sg.n_slices = s1 - s0;
+        sg.c1 = min(P.n_ct, s1 * 8);                                     // a slice is eight column tiles
+        sg.ct0 = s0 * 8 + j0;
+        sg.n_my = sg.ct0 < sg.c1 ? (sg.c1 - sg.ct0 + n_same - 1) / n_same : 0;
+        sg.wsrc = P.tiles + (size_t)(sg.rt * P.K + k) * P.n_ct * 32 + sg.ct0 * 32 + lane;
+        return sg;
+    };
+    auto prefill = [&](const Segment& sg) {                              // the first kRing - 1 tiles of the warp; weights never depend on the stream's past
+#pragma unroll
+        for (int i = 0; i < kRing - 1; ++i) copy_async_16(ring + i * 512, sg.wsrc + (size_t)i * n_same * 32, i < sg.n_my);
+    };
+    bool more = u < u_end;
+    Segment sg;
+    if (more) {
+        sg = next_segment();
+        prefill(sg);
+    }
+    while (more) {
+        const int rt = sg.rt, c1 = sg.c1, ct0 = sg.ct0, n_my = sg.n_my;
+        const uint4* wsrc = sg.wsrc;
         float acc[8][NH][4];
 #pragma unroll
         for (int p = 0; p < 8; ++p)
@@ -112,77 +190,66 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[p][hf][e] = 0.f;
 
-        auto fetch_w = [&](int ct) {                                     // weights: never depend on the stream's past
-            return ldg_stream(P.tiles + (((size_t)rt * P.K + k) * P.n_ct + ct) * 32 + lane);
-        };
-        auto fetch_hx = [&](int ct, Feed<NH>& f) {                       // input scales and activations of the lane's columns (L1 / L2 hits)
-            const __half* hp = P.h + (size_t)k * P.N + ct * 32 + 4 * tq;
-            f.h[0] = __ldg(reinterpret_cast<const uint2*>(hp));
-            f.h[1] = __ldg(reinterpret_cast<const uint2*>(hp + 16));
+        // input scales and activations of the lane's four columns of k-step kh of column tile ct, as loaded (columns 0,1 | 2,3)
+        auto fetch_hx = [&](int ct, int kh, uint2& fh, uint2 (&fx)[NH]) {
+            const int off = ct * 32 + 16 * kh;
+            fh = __ldg(reinterpret_cast<const uint2*>(P.h + hk + off));
 #pragma unroll
-            for (int hf = 0; hf < NH; ++hf) {
-                const int b = 8 * hf + gq;
-                f.x[0][hf] = make_uint2(0u, 0u);
-                f.x[1][hf] = make_uint2(0u, 0u);
-                if (b < P.batch) {
-                    const __half* xp = P.x + (size_t)b * P.N + ct * 32 + 4 * tq;
-                    f.x[0][hf] = __ldcg(reinterpret_cast<const uint2*>(xp));
-                    f.x[1][hf] = __ldcg(reinterpret_cast<const uint2*>(xp + 16));
-                }
-            }
+            for (int hf = 0; hf < NH; ++hf) fx[hf] = __ldcg(reinterpret_cast<const uint2*>(P.x + xb[hf] + off));
         };
 
-        // weights DEPTH tiles ahead (HBM latency), scales and activations one ahead
-        uint4 wq[DEPTH];
-        const int ct0 = c0 + j0;
-#pragma unroll
-        for (int d = 0; d < DEPTH; ++d) {
-            wq[d] = make_uint4(0u, 0u, 0u, 0u);
-            if (ct0 + d * n_same < c1) wq[d] = fetch_w(ct0 + d * n_same);
-        }
+        // weights kRing - 1 tiles ahead (HBM latency), scales and activations one tile ahead, k-step by k-step in place
         if (!waited) {
             asm volatile("griddepcontrol.wait;" ::: "memory");            // x, y and the accumulate words only after this
             waited = true;
         }
-        Feed<NH> cur, nxt;
-        if (ct0 < c1) fetch_hx(ct0, cur);
-        for (int base = ct0; base < c1; base += DEPTH * n_same) {
+        uint2 fh[2], fx[2][NH];
 #pragma unroll
-            for (int d = 0; d < DEPTH; ++d) {
-                const int ct = base + d * n_same;
-                if (ct >= c1) break;
-                const uint4 wv = wq[d];
-                if (ct + DEPTH * n_same < c1) wq[d] = fetch_w(ct + DEPTH * n_same);
-                if (ct + n_same < c1) fetch_hx(ct + n_same, nxt);
+        for (int kh = 0; kh < 2; ++kh) fetch_hx(min(ct0, P.n_ct - 1), kh, fh[kh], fx[kh]);
+        for (int i = 0; i < n_my; ++i) {
+            {
+                const int ct = ct0 + i * n_same;
+                const int ia = i + kRing - 1;                            // the tile that takes the slot freed in the last round
+                copy_async_16(ring + (ia & (kRing - 1)) * 512, wsrc + (size_t)ia * n_same * 32, ia < n_my);
+                copy_async_wait<kRing - 1>();                            // tile i has landed (one group per tile, also for the tiles that do not exist)
+                const uint4 wv = lds_128(ring + (i & (kRing - 1)) * 512);
+                const int ct_next = min(ct + n_same, P.n_ct - 1);        // beyond the segment: a valid address, never used
                 const uint32_t w[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
                 for (int kh = 0; kh < 2; ++kh) {
-                    const uint32_t h01 = cur.h[kh].x, h23 = cur.h[kh].y;
+                    const uint32_t h02 = prmt(fh[kh].x, fh[kh].y, 0x5410), h13 = prmt(fh[kh].x, fh[kh].y, 0x7632);
+                    uint32_t b0[NH], b1[NH];
 #pragma unroll
-                    for (int p = 0; p < 8; ++p) {
-                        const uint32_t sl = w[2 * kh] << (7 - p), sh = w[2 * kh + 1] << (7 - p);   // bit p of every byte -> bit 7
-                        const uint32_t a0 = flip(prmt(sl, 0u, 0x1404), h01), a2 = flip(prmt(sl, 0u, 0x3424), h23);
-                        const uint32_t a1 = flip(prmt(sh, 0u, 0x1404), h01), a3 = flip(prmt(sh, 0u, 0x3424), h23);
+                    for (int hf = 0; hf < NH; ++hf) {
+                        b0[hf] = prmt(fx[kh][hf].x, fx[kh][hf].y, 0x5410);
+                        b1[hf] = prmt(fx[kh][hf].x, fx[kh][hf].y, 0x7632);
+                    }
+                    fetch_hx(ct_next, kh, fh[kh], fx[kh]);                // the same k-step of the warp's next tile, in place
+                    // u = w * 2^(7-p): bit p of bytes 1 and 3 -> bits 15 and 31;  v = u * 2^8: the same for bytes 0 and 2
+                    uint32_t ul = w[2 * kh], uh = w[2 * kh + 1];
+                    uint32_t vl = mul_lo(ul, P.two_pow_8), vh = mul_lo(uh, P.two_pow_8);
 #pragma unroll
-                        for (int hf = 0; hf < NH; ++hf) mma_f16(acc[p][hf], a0, a1, a2, a3, cur.x[kh][hf].x, cur.x[kh][hf].y);
+                    for (int p = 7; p >= 0; --p) {
+                        const uint32_t a0 = flip(vl, h02), a1 = flip(vh, h02), a2 = flip(ul, h13), a3 = flip(uh, h13);
+#pragma unroll
+                        for (int hf = 0; hf < NH; ++hf) mma_f16(acc[p][hf], a0, a1, a2, a3, b0[hf], b1[hf]);
+                        if (p > 0) {
+                            ul = mul_lo(ul, P.two); uh = mul_lo(uh, P.two);
+                            vl = mul_lo(vl, P.two); vh = mul_lo(vh, P.two);
+                        }
                     }
                 }
-                cur = nxt;
             }
         }
-        // the path's output scale, in place
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            const int row = rt * RABIT_TILE_ROWS + 16 * p + gq;
-            const float g_lo = __half2float(P.g[(size_t)k * P.Mp + row]), g_hi = __half2float(P.g[(size_t)k * P.Mp + row + 8]);
-#pragma unroll
-            for (int hf = 0; hf < NH; ++hf) {
-                acc[p][hf][0] *= g_lo; acc[p][hf][1] *= g_lo;
-                acc[p][hf][2] *= g_hi; acc[p][hf][3] *= g_hi;
-            }
+        copy_async_wait<0>();
+        // the next segment's first tiles set off now: they cross HBM while this segment is added up
+        const int n_slices = sg.n_slices;
+        more = u < u_end;
+        if (more) {
+            sg = next_segment();
+            prefill(sg);
         }
-
-        // ---- the warp's scaled partial outputs -> its slot; slot layout [batch row][row of the tile]
+        // ---- the warp's partial outputs -> its slot; slot layout [batch row][row of the tile]
         float* mine = slots + (size_t)warp * (NH * 8 * 128);
 #pragma unroll
         for (int p = 0; p < 8; ++p)
@@ -195,19 +262,26 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
                 mine[(b + 1) * 128 + row + 8] = acc[p][hf][3];
             }
         __syncthreads();
-        // ---- fixed-order sum over the warps, then one atomic per output of the unit
-        const int n_slices = s1 - s0;
+        // ---- fixed-order sum over the warps, then one atomic per output of the segment
+        const int arrivals = owner_of((long long)(rt + 1) * P.n_cs - 1, P.n_pairs, gridDim.x) -
+                             owner_of((long long)rt * P.n_cs, P.n_pairs, gridDim.x) + 1;    // segments of this row tile
         constexpr int kPer = NH * 8 * 128 / kThreads;                    // outputs per thread (4 or 8)
         unsigned long long old[kPer], add[kPer];
         bool bad[kPer];
+        __half gk[kPer][RABIT_MAX_K];                                     // output scales of the thread's rows: all loads in flight together
+#pragma unroll
+        for (int i = 0; i < kPer; ++i)
+#pragma unroll
+            for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+                gk[i][kk] = kk < P.K ? P.g[(size_t)kk * P.Mp + rt * RABIT_TILE_ROWS + ((tid + i * kThreads) & 127)] : __half();
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
             const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
             old[i] = 0ULL; add[i] = 0ULL; bad[i] = false;
             if (b >= P.batch) continue;
-            float v = 0.f;
-#pragma unroll
-            for (int wv = 0; wv < kWarps; ++wv) v += slots[(size_t)wv * (NH * 8 * 128) + o];
+            // sum_k g_k * (sum over the warps of path k), in a fixed order
+            const float* col = slots + o;
+            const float v = P.K == 2 ? path_sums<2, NH>(col, gk[i]) : P.K == 3 ? path_sums<3, NH>(col, gk[i]) : path_sums<1, NH>(col, gk[i]);
             const float scaled = v * P.inv_unit;
             bad[i] = !(fabsf(scaled) < P.limit * (float)n_slices);       // inf or NaN: finite inputs cannot get here
             const long long q = bad[i] ? 0LL : __float2ll_rn(scaled);
@@ -220,7 +294,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         for (int i = 0; i < kPer; ++i) {
             const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
             if (b >= P.batch) continue;
-            if ((int)((old[i] >> 55) & 0xFFu) != P.splits - 1) continue;  // other column ranges are still to come
+            if ((int)((old[i] >> 55) & 0xFFu) != arrivals - 1) continue;  // other segments of the row tile are still to come
             const unsigned long long sum = (old[i] & kSumMask) + (add[i] & kSumMask);
             const long long total = (long long)sum - ((long long)P.n_cs << P.fix_bits);
             const bool poisoned = bad[i] || (old[i] >> 63) != 0;
@@ -229,18 +303,18 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             if (row < P.M) P.y[(size_t)b * P.M + row] = __float2half_rn(v);
             P.acc[(size_t)b * P.Mp + row] = 0ULL;                         // resting state for the next call
         }
-        __syncthreads();                                                 // the slots are free for the next unit
+        __syncthreads();                                                 // the slots are free for the next segment
     }
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-template <int NH, int DEPTH>
+template <int NH>
 cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream) {
     static bool attr_done[64] = {false};
-    const size_t smem = (size_t)kWarps * NH * 8 * 128 * sizeof(float);
+    const size_t smem = (size_t)kWarps * NH * 8 * 128 * sizeof(float) + (size_t)kWarps * kRing * 512;
     const int slot = device >= 0 && device < 64 ? device : 0;
     if (!attr_done[slot] || slot != device) {
-        cudaError_t e = cudaFuncSetAttribute(rabit_gemv_f16_kernel<NH, DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(rabit_gemv_f16_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done[slot] = true;
     }
@@ -254,7 +328,7 @@ cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rabit_gemv_f16_kernel<NH, DEPTH>, P);
+    return cudaLaunchKernelEx(&cfg, rabit_gemv_f16_kernel<NH>, P);
 }
 
 }  // namespace
@@ -262,7 +336,8 @@ cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream
 bool rabit_gemv_f16_supports(const rabit_layer& L, int batch) {
     if (batch < 1 || batch > RABIT_MAX_GEMV_BATCH) return false;
     if (L.geom.n_cs > RABIT_LUT_MAX_SLICES || L.d_acc == nullptr) return false;
-    return (long long)L.geom.n_rt * L.geom.n_cs < kMaxUnits;
+    if ((long long)L.geom.n_rt * L.geom.K * L.geom.n_ct * 32 >= (1LL << 31)) return false;   // 32-bit tile offsets in the kernel
+    return (long long)L.geom.n_rt * L.geom.n_cs < kMaxPairs;
 }
 
 // One launch, 1..16 batch rows (x: [batch][N], y: [batch][M]).
@@ -282,20 +357,11 @@ cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, 
     P.unit = ldexpf(1.f, G.unit_exp);
     P.inv_unit = ldexpf(1.f, -G.unit_exp);
     P.limit = ldexpf(1.f, G.fix_bits);
+    P.two = 2u;
+    P.two_pow_8 = 256u;
+    P.n_pairs = G.n_rt * G.n_cs;
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
     const int resident = 2 * sms;                                        // two CTAs per SM
-    // Column ranges per row tile: the split that minimises  waves x (slices per unit + 1)  (a unit's fixed cost, its
-    // reduction and atomics, is about one slice's worth of tiles).
-    int splits = 1;
-    long long best = -1;
-    for (int s = 1; s <= G.n_cs; ++s) {
-        const long long units = (long long)G.n_rt * s;
-        const long long waves = (units + resident - 1) / resident;
-        const long long cost = waves * ((G.n_cs + s - 1) / s + 1);
-        if (best < 0 || cost < best) { best = cost; splits = s; }
-    }
-    P.splits = splits;
-    P.n_units = G.n_rt * splits;
-    const int grid = P.n_units < resident ? P.n_units : resident;
-    return batch <= 8 ? launch<1, 4>(P, grid, L.device, stream) : launch<2, 2>(P, grid, L.device, stream);
+    const int grid = P.n_pairs < resident ? P.n_pairs : resident;
+    return batch <= 8 ? launch<1>(P, grid, L.device, stream) : launch<2>(P, grid, L.device, stream);
 }
