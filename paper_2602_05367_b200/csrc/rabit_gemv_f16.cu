@@ -42,6 +42,7 @@
 
 #include <algorithm>
 #include <cstring>
+#include <vector>
 
 #include "rabit_internal.h"
 
@@ -51,6 +52,8 @@ constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRing = 8;                               // sign tiles a warp keeps in flight or in use (a power of two)
 constexpr long long kMaxPairs = 1LL << 30;
+constexpr int kMaxGrid = 2 * 160;                     // two CTAs per SM, up to 160 SMs
+constexpr int kSlotStride = 128 + 4;                  // floats per batch row of a slot: the pad spreads a warp's store over all banks
 constexpr unsigned long long kSumMask = (1ULL << 55) - 1;
 
 struct F16Params {
@@ -62,10 +65,11 @@ struct F16Params {
     unsigned long long* acc;        // [16][Mp], all zero between calls
     int K, M, N, Mp, n_rt, n_ct, n_cs;
     int batch;
-    int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; CTA c owns pairs [c * n_pairs / grid, (c + 1) * n_pairs / grid)
+    int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; CTA c owns pairs [bound[c], bound[c + 1])
     int fix_bits;
     float inv_unit, unit, limit;
     uint32_t two, two_pow_8;        // 2 and 256: multipliers the compiler cannot fold into shifts
+    int bound[kMaxGrid + 1];        // ascending; bound[grid] = n_pairs
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
@@ -113,27 +117,33 @@ __device__ __forceinline__ float path_sums(const float* col, const __half (&g)[R
 #pragma unroll
     for (int kk = 0; kk < KK; ++kk) sk[kk] = 0.f;
 #pragma unroll
-    for (int wv = 0; wv < kWarps; ++wv) sk[wv % KK] += col[(size_t)wv * (NH * 8 * 128)];
+    for (int wv = 0; wv < kWarps; ++wv) sk[wv % KK] += col[(size_t)wv * (NH * 8 * kSlotStride)];
     float v = 0.f;
 #pragma unroll
     for (int kk = 0; kk < KK; ++kk) v = fmaf(__half2float(g[kk]), sk[kk], v);
     return v;
 }
 
-// First CTA whose range holds pair u:  the largest c with  c * n_pairs / grid <= u.
-__device__ __forceinline__ int owner_of(long long u, int n_pairs, int grid) {
-    return (int)(((u + 1) * grid - 1) / n_pairs);
+// The CTA whose range holds pair u: the last c with bound[c] <= u (empty ranges have bound[c] == bound[c + 1] and lose to
+// the non-empty one that follows them).
+__device__ __forceinline__ int owner_of(const F16Params& P, int u, int grid) {
+    int lo = 0, hi = grid - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (P.bound[mid] <= u) lo = mid; else hi = mid - 1;
+    }
+    return lo;
 }
 
 // NH = halves of the batch (8 rows each) a pass carries.
 template <int NH>
 __global__ void __launch_bounds__(kThreads, 2)
 rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
-    extern __shared__ __align__(16) float slots[];                       // [kWarps][NH * 8][128] scaled partial outputs, then the rings
+    extern __shared__ __align__(16) float slots[];                       // [kWarps][NH * 8][kSlotStride] partial outputs, then the rings
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tq = lane & 3;
     // the lane's 16 bytes of ring slot 0 of its warp; slot r is r * 512 bytes further
-    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(slots) + (uint32_t)(kWarps * NH * 8 * 128 * sizeof(float)) +
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(slots) + (uint32_t)(kWarps * NH * 8 * kSlotStride * sizeof(float)) +
                           (uint32_t)((warp * kRing * 32 + lane) * 16);
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -154,13 +164,13 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         int rt, n_slices, c1, ct0, n_my;
         const uint4* wsrc;                                               // the warp's first tile (this lane's 16 bytes)
     };
-    long long u = (long long)blockIdx.x * P.n_pairs / gridDim.x;
-    const long long u_end = (long long)(blockIdx.x + 1) * P.n_pairs / gridDim.x;
+    int u = P.bound[blockIdx.x];
+    const int u_end = P.bound[blockIdx.x + 1];
     auto next_segment = [&]() {                                          // the segment that starts at pair u; advances u
         Segment sg;
-        sg.rt = (int)(u / P.n_cs);
-        const int s0 = (int)(u - (long long)sg.rt * P.n_cs);
-        const int s1 = (int)min((long long)P.n_cs, s0 + (u_end - u));
+        sg.rt = u / P.n_cs;
+        const int s0 = u - sg.rt * P.n_cs;
+        const int s1 = min(P.n_cs, s0 + (u_end - u));
         u += s1 - s0;
         sg.n_slices = s1 - s0;
         sg.c1 = min(P.n_ct, s1 * 8);                                     // a slice is eight column tiles
@@ -180,7 +190,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         prefill(sg);
     }
     while (more) {
-        const int rt = sg.rt, c1 = sg.c1, ct0 = sg.ct0, n_my = sg.n_my;
+        const int rt = sg.rt, ct0 = sg.ct0, n_my = sg.n_my;
         const uint4* wsrc = sg.wsrc;
         float acc[8][NH][4];
 #pragma unroll
@@ -249,45 +259,49 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             sg = next_segment();
             prefill(sg);
         }
+        constexpr int kPer = NH * 8 * 128 / kThreads;                    // outputs per thread (4 or 8)
+        __half gk[RABIT_MAX_K];                                           // output scales of the thread's row (the same row for all its outputs), loaded early
+#pragma unroll
+        for (int kk = 0; kk < RABIT_MAX_K; ++kk)
+            gk[kk] = kk < P.K ? P.g[(size_t)kk * P.Mp + rt * RABIT_TILE_ROWS + (tid & 127)] : __half();
         // ---- the warp's partial outputs -> its slot; slot layout [batch row][row of the tile]
-        float* mine = slots + (size_t)warp * (NH * 8 * 128);
+        float* mine = slots + (size_t)warp * (NH * 8 * kSlotStride);
 #pragma unroll
         for (int p = 0; p < 8; ++p)
 #pragma unroll
             for (int hf = 0; hf < NH; ++hf) {
                 const int b = 8 * hf + 2 * tq, row = 16 * p + gq;
-                mine[(b) * 128 + row] = acc[p][hf][0];
-                mine[(b + 1) * 128 + row] = acc[p][hf][1];
-                mine[(b) * 128 + row + 8] = acc[p][hf][2];
-                mine[(b + 1) * 128 + row + 8] = acc[p][hf][3];
+                mine[(b) * kSlotStride + row] = acc[p][hf][0];
+                mine[(b + 1) * kSlotStride + row] = acc[p][hf][1];
+                mine[(b) * kSlotStride + row + 8] = acc[p][hf][2];
+                mine[(b + 1) * kSlotStride + row + 8] = acc[p][hf][3];
             }
         __syncthreads();
         // ---- fixed-order sum over the warps, then one atomic per output of the segment
-        const int arrivals = owner_of((long long)(rt + 1) * P.n_cs - 1, P.n_pairs, gridDim.x) -
-                             owner_of((long long)rt * P.n_cs, P.n_pairs, gridDim.x) + 1;    // segments of this row tile
-        constexpr int kPer = NH * 8 * 128 / kThreads;                    // outputs per thread (4 or 8)
+        const int arrivals = owner_of(P, (rt + 1) * P.n_cs - 1, gridDim.x) - owner_of(P, rt * P.n_cs, gridDim.x) + 1;   // segments of this row tile
+        // (thread t owns row t & 127 of the tile and the batch rows (t >> 7) + 2 i; rows beyond the batch are computed from
+        // whatever their MMA columns held and dropped)
         unsigned long long old[kPer], add[kPer];
         bool bad[kPer];
-        __half gk[kPer][RABIT_MAX_K];                                     // output scales of the thread's rows: all loads in flight together
-#pragma unroll
-        for (int i = 0; i < kPer; ++i)
-#pragma unroll
-            for (int kk = 0; kk < RABIT_MAX_K; ++kk)
-                gk[i][kk] = kk < P.K ? P.g[(size_t)kk * P.Mp + rt * RABIT_TILE_ROWS + ((tid + i * kThreads) & 127)] : __half();
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
             const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
-            old[i] = 0ULL; add[i] = 0ULL; bad[i] = false;
-            if (b >= P.batch) continue;
             // sum_k g_k * (sum over the warps of path k), in a fixed order
-            const float* col = slots + o;
-            const float v = P.K == 2 ? path_sums<2, NH>(col, gk[i]) : P.K == 3 ? path_sums<3, NH>(col, gk[i]) : path_sums<1, NH>(col, gk[i]);
+            const float* col = slots + b * kSlotStride + rl;
+            const float v = P.K == 2 ? path_sums<2, NH>(col, gk) : P.K == 3 ? path_sums<3, NH>(col, gk) : path_sums<1, NH>(col, gk);
             const float scaled = v * P.inv_unit;
             bad[i] = !(fabsf(scaled) < P.limit * (float)n_slices);       // inf or NaN: finite inputs cannot get here
             const long long q = bad[i] ? 0LL : __float2ll_rn(scaled);
             add[i] = (unsigned long long)(q + ((long long)n_slices << P.fix_bits)) + (1ULL << 55);
+        }
+        // all atomics of the thread back to back: nothing between them that could wait for an answer
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
+            old[i] = 0ULL;
+            if (b >= P.batch) continue;
             unsigned long long* word = P.acc + (size_t)b * P.Mp + rt * RABIT_TILE_ROWS + rl;
-            if (bad[i]) atomicOr(word, 1ULL << 63);
+            if (bad[i]) atomicOr(word, 1ULL << 63);                      // sticky: the add below never carries into bit 63
             old[i] = atomicAdd(word, add[i]);
         }
 #pragma unroll
@@ -311,7 +325,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
 template <int NH>
 cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream) {
     static bool attr_done[64] = {false};
-    const size_t smem = (size_t)kWarps * NH * 8 * 128 * sizeof(float) + (size_t)kWarps * kRing * 512;
+    const size_t smem = (size_t)kWarps * NH * 8 * kSlotStride * sizeof(float) + (size_t)kWarps * kRing * 512;
     const int slot = device >= 0 && device < 64 ? device : 0;
     if (!attr_done[slot] || slot != device) {
         cudaError_t e = cudaFuncSetAttribute(rabit_gemv_f16_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -329,6 +343,71 @@ cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, rabit_gemv_f16_kernel<NH>, P);
+}
+
+}  // namespace
+
+namespace {
+
+// Cuts the n_rt * n_cs (row tile, slice) pairs, in that order, into at most `resident` contiguous ranges of about equal
+// COST, where a range costs one unit per pair plus `seg` units per segment (per row tile it touches): the end of a segment
+// (adding up the warps, the atomics and their answers) takes a CTA as long as two to three slices of MMAs.  So a range that
+// spans a row-tile boundary gets fewer pairs, and no range starts a row tile it cannot spend at least one pair on.  The
+// smallest per-range cost limit that needs no more than `resident` ranges is found by bisection; bound[] receives the
+// range starts (bound[grid] = n_pairs).  Returns the number of ranges.  Plans are cached per thread.
+int plan_ranges(int n_rt, int n_cs, int K, int NH, int resident, int* bound) {
+    struct Plan { int n_rt, n_cs, K, NH, resident, grid; int bound[kMaxGrid + 1]; };
+    static thread_local std::vector<Plan> plans;
+    for (const Plan& pl : plans)
+        if (pl.n_rt == n_rt && pl.n_cs == n_cs && pl.K == K && pl.NH == NH && pl.resident == resident) {
+            std::memcpy(bound, pl.bound, sizeof(pl.bound));
+            return pl.grid;
+        }
+    // fitted to timelines on B200: a pair is 8 K tiles at about 0.07 (NH = 1) or 0.085 us (NH = 2) each per CTA, a segment end 3 to 4 us
+    const double seg = (NH == 1 ? 3.0 : 4.0) / (8.0 * K * (NH == 1 ? 0.07 : 0.085));
+    const long long n_pairs = (long long)n_rt * n_cs;
+    auto cut = [&](double limit, int* out) {                             // greedy walk; returns the number of ranges (may exceed resident: then out is not filled further)
+        int n = 0;
+        long long u = 0;
+        while (u < n_pairs) {
+            if (n < resident && out) out[n] = (int)u;
+            ++n;
+            if (n > resident && !out) return n;
+            double c = 0.0;
+            bool first = true;
+            while (u < n_pairs) {
+                const long long left = n_cs - u % n_cs;                  // pairs to the end of this row tile
+                long long take = (long long)(limit - c - seg);           // pairs the budget still pays for after the segment's end
+                if (take < 1) {
+                    if (!first) break;                                   // do not start a segment the range cannot use
+                    take = 1;
+                }
+                if (take > left) take = left;
+                u += take;
+                c += seg + (double)take;
+                first = false;
+            }
+        }
+        return n;
+    };
+    double lo = seg + 1.0, hi = seg * (n_rt + 1) + (double)n_pairs + 1.0;
+    if (cut(lo, nullptr) > resident) {
+        for (int it = 0; it < 48; ++it) {
+            const double mid = 0.5 * (lo + hi);
+            if (cut(mid, nullptr) <= resident) hi = mid; else lo = mid;
+        }
+    } else {
+        hi = lo;
+    }
+    int tmp[kMaxGrid + 1];
+    const int grid = cut(hi, tmp);
+    for (int c = 0; c <= kMaxGrid; ++c) bound[c] = c < grid ? tmp[c] : (int)n_pairs;
+    if (plans.size() >= 256) plans.clear();
+    plans.emplace_back();
+    Plan& pl = plans.back();
+    pl.n_rt = n_rt; pl.n_cs = n_cs; pl.K = K; pl.NH = NH; pl.resident = resident; pl.grid = grid;
+    std::memcpy(pl.bound, bound, sizeof(pl.bound));
+    return grid;
 }
 
 }  // namespace
@@ -361,7 +440,7 @@ cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, 
     P.two_pow_8 = 256u;
     P.n_pairs = G.n_rt * G.n_cs;
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
-    const int resident = 2 * sms;                                        // two CTAs per SM
-    const int grid = P.n_pairs < resident ? P.n_pairs : resident;
+    const int resident = std::min(2 * sms, kMaxGrid);                    // two CTAs per SM
+    const int grid = plan_ranges(G.n_rt, G.n_cs, G.K, batch > 8 ? 2 : 1, resident, P.bound);
     return batch <= 8 ? launch<1>(P, grid, L.device, stream) : launch<2>(P, grid, L.device, stream);
 }
