@@ -484,7 +484,7 @@ def bench_extras(args, rabit, device, stream, shapes, layers, peaks) -> dict:
                                             "note": "one token = one CUDA graph of %d launches (plus three tiny launches that select the token's "
                                                     "activations by a device-side index); tokens/s = 256 / elapsed" % (len(layers) * len(GROUPS))}
 
-    # config 3 / 4 samples at batch 1, batch 16 on the 8B shapes, the batch-512 GEMM, and K = 1 / 3 at 7B shapes
+    # config 3 / 4 samples at batch 1, batches 1, 8 and 16 on the 8B shapes, the batch-512 GEMM, and K = 1 / 3 at 7B shapes
     extra_hbm = []
     for (M, N) in [(14336, 4096), (28672, 8192)]:
         lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 4)
@@ -505,14 +505,14 @@ def bench_extras(args, rabit, device, stream, shapes, layers, peaks) -> dict:
     b16 = []
     for (M, N) in [(4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336)]:
         lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 3)
-        for batch in (1, 16):
+        for batch in (1, 8, 16):
             x = torch.from_numpy(make_x(batch, N, key=(3, batch, N))).to(device)
             y = torch.zeros((batch, M), dtype=torch.float16, device=device)
             b16.append(hbm_case(M, N, K_PATHS, batch, timed_case(lys, x, y)))
         for L in lys:
             L.free()
         del lys
-    out["llama3_8b_shapes_batch_1_and_16"] = b16
+    out["llama3_8b_shapes_batch_1_8_16"] = b16
     kk = []
     for K in (1, 3):
         for (M, N) in [(4096, 4096), (11008, 4096)]:

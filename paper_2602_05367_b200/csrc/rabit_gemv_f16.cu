@@ -24,20 +24,21 @@
 // and the accumulator lane holds rows gq, gq + 8 of the block and batch rows 2tq, 2tq + 1.
 //
 // Work split.  The layer is n_rt row tiles x n_cs slices of 256 columns; in that order the (row tile, slice) pairs are cut
-// into one contiguous range per CTA, all the same length to within one pair.  The part of a range inside one row tile is a
-// segment.  CTAs of 8 warps, two per SM (while one adds up a segment and waits for its atomics the other computes; one
-// CTA of 16 warps per SM measured 15 % slower); warp w works on path w % K and shares the column tiles of the segment with the other warps
-// of that path.  A warp streams its tiles through a ring of its own in shared memory with asynchronous 16-byte copies
-// (one per lane and tile, each lane reads back only what it copied itself, so no barrier is involved), kRing - 1 tiles
-// ahead: with 16 warps per SM that keeps about 56 KB per SM in flight, which is what the HBM latency needs (with the
-// tiles prefetched into registers, two to four per warp, the kernel ran at the speed of its memory latency, 1.1 to
-// 1.7 TB/s).  At the end of a segment every warp writes
-// its accumulators to its own slot of shared memory, the CTA adds the slots path by path in a fixed order (deterministic)
-// and applies g_k to each path's sum, and every output of the segment goes, as in the table-driven kernel, into the row's 64-bit accumulate
-// word with one integer atomic (fixed-point grid of the packer, arrival count in bits 55..62, bit 63 = non-finite); the
-// lane whose add completes a row (the count reaches the number of segments of that row tile) rounds it to fp16, stores y
-// and clears the word.  A contribution that covers s slices is shifted by s * 2^fix_bits, so the total shift is the same
-// n_cs * 2^fix_bits for every split.  Nothing waits for another CTA.
+// into one contiguous range per SM, all the same length to within one pair, and every SM's range into two parts.  One
+// CTA of 16 warps per SM; its two groups of 8 warps each take one part and share nothing but the SM (own barrier, own
+// shared memory): while one group adds up a segment and waits for its atomics, the other computes.  The part of a range
+// inside one row tile is a segment.  Warp w of a group works on path w % K and shares the column tiles of the segment
+// with the other warps of that path.  A warp streams its tiles through a ring of its own in shared memory with
+// asynchronous 16-byte copies (one per lane and tile, each lane reads back only what it copied itself, so no barrier is
+// involved), kRing - 1 tiles ahead: with 16 warps per SM that keeps about 56 KB per SM in flight, which is what the HBM
+// latency needs (with the tiles prefetched into registers, two to four per warp, the kernel ran at the speed of its
+// memory latency, 1.1 to 1.7 TB/s).  At the end of a segment every warp writes its accumulators to its own slot of shared
+// memory, the group adds the slots path by path in a fixed order (deterministic) and applies g_k to each path's sum, and
+// every output of the segment goes, as in the table-driven kernel, into the row's 64-bit accumulate word with one
+// integer atomic (fixed-point grid of the packer, arrival count in bits 55..62, bit 63 = non-finite); the thread whose
+// add completes a row (the count reaches the number of segments of that row tile) rounds it to fp16, stores y and clears
+// the word.  A contribution that covers s slices is shifted by s * 2^fix_bits, so the total shift is the same
+// n_cs * 2^fix_bits for every split.  Nothing waits for another CTA or for the other group.
 #include <cuda_fp16.h>
 
 #include <algorithm>
@@ -48,11 +49,13 @@
 
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
+constexpr int kWarps = 8;                              // warps of a group
+constexpr int kGroupThreads = kWarps * 32;
+constexpr int kGroups = 2;                             // independent groups of a CTA (one CTA per SM)
+constexpr int kThreads = kGroups * kGroupThreads;
 constexpr int kRing = 8;                               // sign tiles a warp keeps in flight or in use (a power of two)
 constexpr long long kMaxPairs = 1LL << 30;
-constexpr int kMaxGrid = 2 * 160;                     // two CTAs per SM, up to 160 SMs
+constexpr int kMaxRanges = kGroups * 160;              // one range per group, up to 160 SMs
 constexpr int kSlotStride = 128 + 4;                  // floats per batch row of a slot: the pad spreads a warp's store over all banks
 constexpr unsigned long long kSumMask = (1ULL << 55) - 1;
 
@@ -65,11 +68,11 @@ struct F16Params {
     unsigned long long* acc;        // [16][Mp], all zero between calls
     int K, M, N, Mp, n_rt, n_ct, n_cs;
     int batch;
-    int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; CTA c owns pairs [bound[c], bound[c + 1])
+    int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; group q of CTA c owns pairs [bound[2c + q], bound[2c + q + 1])
     int fix_bits;
     float inv_unit, unit, limit;
     uint32_t two, two_pow_8;        // 2 and 256: multipliers the compiler cannot fold into shifts
-    int bound[kMaxGrid + 1];        // ascending; bound[grid] = n_pairs
+    int bound[kMaxRanges + 1];      // ascending; bound[2 * grid] = n_pairs
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
@@ -103,6 +106,10 @@ template <int N>
 __device__ __forceinline__ void copy_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
+// barrier of one group (ids 1 and 2; 0 is left to __syncthreads)
+__device__ __forceinline__ void group_sync(int group) {
+    asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "n"(kGroupThreads) : "memory");
+}
 __device__ __forceinline__ uint4 lds_128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
@@ -124,10 +131,10 @@ __device__ __forceinline__ float path_sums(const float* col, const __half (&g)[R
     return v;
 }
 
-// The CTA whose range holds pair u: the last c with bound[c] <= u (empty ranges have bound[c] == bound[c + 1] and lose to
+// The range that holds pair u: the last r with bound[r] <= u (empty ranges have bound[r] == bound[r + 1] and lose to
 // the non-empty one that follows them).
-__device__ __forceinline__ int owner_of(const F16Params& P, int u, int grid) {
-    int lo = 0, hi = grid - 1;
+__device__ __forceinline__ int owner_of(const F16Params& P, int u, int n_ranges) {
+    int lo = 0, hi = n_ranges - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         if (P.bound[mid] <= u) lo = mid; else hi = mid - 1;
@@ -137,11 +144,14 @@ __device__ __forceinline__ int owner_of(const F16Params& P, int u, int grid) {
 
 // NH = halves of the batch (8 rows each) a pass carries.
 template <int NH>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
-    extern __shared__ __align__(16) float slots[];                       // [kWarps][NH * 8][kSlotStride] partial outputs, then the rings
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    extern __shared__ __align__(16) float smem_f[];                      // per group: [kWarps][NH * 8][kSlotStride] partial outputs, then the warps' rings
+    constexpr int kGroupFloats = kWarps * NH * 8 * kSlotStride + kWarps * kRing * 128;
+    const int group = threadIdx.x / kGroupThreads;                       // the two groups share nothing but the SM
+    const int tid = threadIdx.x % kGroupThreads, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tq = lane & 3;
+    float* slots = smem_f + (size_t)group * kGroupFloats;
     // the lane's 16 bytes of ring slot 0 of its warp; slot r is r * 512 bytes further
     const uint32_t ring = (uint32_t)__cvta_generic_to_shared(slots) + (uint32_t)(kWarps * NH * 8 * kSlotStride * sizeof(float)) +
                           (uint32_t)((warp * kRing * 32 + lane) * 16);
@@ -149,8 +159,8 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool waited = false;
 
-    // every warp works on ONE path: path k = warp % K, and the column tiles of a segment are dealt out among the warps of
-    // that path (K = 3: three, three and two warps)
+    // every warp works on ONE path: path k = warp % K, and the column tiles of a segment are dealt out among the group's
+    // warps of that path (K = 3: three, three and two warps)
     const int k = warp % P.K;
     const int n_same = (kWarps - k + P.K - 1) / P.K, j0 = warp / P.K;
     const int hk = k * P.N + 4 * tq;                                      // element offsets (K * N and 16 * N fit 31 bits: N <= 65280)
@@ -164,8 +174,9 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         int rt, n_slices, c1, ct0, n_my;
         const uint4* wsrc;                                               // the warp's first tile (this lane's 16 bytes)
     };
-    int u = P.bound[blockIdx.x];
-    const int u_end = P.bound[blockIdx.x + 1];
+    const int n_ranges = kGroups * gridDim.x;
+    int u = P.bound[kGroups * blockIdx.x + group];
+    const int u_end = P.bound[kGroups * blockIdx.x + group + 1];
     auto next_segment = [&]() {                                          // the segment that starts at pair u; advances u
         Segment sg;
         sg.rt = u / P.n_cs;
@@ -259,7 +270,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             sg = next_segment();
             prefill(sg);
         }
-        constexpr int kPer = NH * 8 * 128 / kThreads;                    // outputs per thread (4 or 8)
+        constexpr int kPer = NH * 8 * 128 / kGroupThreads;                    // outputs per thread (4 or 8)
         __half gk[RABIT_MAX_K];                                           // output scales of the thread's row (the same row for all its outputs), loaded early
 #pragma unroll
         for (int kk = 0; kk < RABIT_MAX_K; ++kk)
@@ -276,16 +287,18 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
                 mine[(b) * kSlotStride + row + 8] = acc[p][hf][2];
                 mine[(b + 1) * kSlotStride + row + 8] = acc[p][hf][3];
             }
-        __syncthreads();
+        group_sync(group);
         // ---- fixed-order sum over the warps, then one atomic per output of the segment
-        const int arrivals = owner_of(P, (rt + 1) * P.n_cs - 1, gridDim.x) - owner_of(P, rt * P.n_cs, gridDim.x) + 1;   // segments of this row tile
+        int arrivals = 0;                                                // segments of this row tile: the non-empty ranges that touch it
+        for (int r = owner_of(P, rt * P.n_cs, n_ranges), r1 = owner_of(P, (rt + 1) * P.n_cs - 1, n_ranges); r <= r1; ++r)
+            arrivals += P.bound[r] < P.bound[r + 1] ? 1 : 0;
         // (thread t owns row t & 127 of the tile and the batch rows (t >> 7) + 2 i; rows beyond the batch are computed from
         // whatever their MMA columns held and dropped)
         unsigned long long old[kPer], add[kPer];
         bool bad[kPer];
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
-            const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
+            const int o = tid + i * kGroupThreads, b = o >> 7, rl = o & 127;
             // sum_k g_k * (sum over the warps of path k), in a fixed order
             const float* col = slots + b * kSlotStride + rl;
             const float v = P.K == 2 ? path_sums<2, NH>(col, gk) : P.K == 3 ? path_sums<3, NH>(col, gk) : path_sums<1, NH>(col, gk);
@@ -297,7 +310,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         // all atomics of the thread back to back: nothing between them that could wait for an answer
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
-            const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
+            const int o = tid + i * kGroupThreads, b = o >> 7, rl = o & 127;
             old[i] = 0ULL;
             if (b >= P.batch) continue;
             unsigned long long* word = P.acc + (size_t)b * P.Mp + rt * RABIT_TILE_ROWS + rl;
@@ -306,7 +319,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         }
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
-            const int o = tid + i * kThreads, b = o >> 7, rl = o & 127;
+            const int o = tid + i * kGroupThreads, b = o >> 7, rl = o & 127;
             if (b >= P.batch) continue;
             if ((int)((old[i] >> 55) & 0xFFu) != arrivals - 1) continue;  // other segments of the row tile are still to come
             const unsigned long long sum = (old[i] & kSumMask) + (add[i] & kSumMask);
@@ -317,7 +330,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             if (row < P.M) P.y[(size_t)b * P.M + row] = __float2half_rn(v);
             P.acc[(size_t)b * P.Mp + row] = 0ULL;                         // resting state for the next call
         }
-        __syncthreads();                                                 // the slots are free for the next segment
+        group_sync(group);                                               // the slots are free for the next segment
     }
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
@@ -325,7 +338,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
 template <int NH>
 cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream) {
     static bool attr_done[64] = {false};
-    const size_t smem = (size_t)kWarps * NH * 8 * kSlotStride * sizeof(float) + (size_t)kWarps * kRing * 512;
+    const size_t smem = (size_t)kGroups * ((size_t)kWarps * NH * 8 * kSlotStride * sizeof(float) + (size_t)kWarps * kRing * 512);
     const int slot = device >= 0 && device < 64 ? device : 0;
     if (!attr_done[slot] || slot != device) {
         cudaError_t e = cudaFuncSetAttribute(rabit_gemv_f16_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -349,64 +362,27 @@ cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream
 
 namespace {
 
-// Cuts the n_rt * n_cs (row tile, slice) pairs, in that order, into at most `resident` contiguous ranges of about equal
-// COST, where a range costs one unit per pair plus `seg` units per segment (per row tile it touches): the end of a segment
-// (adding up the warps, the atomics and their answers) takes a CTA as long as two to three slices of MMAs.  So a range that
-// spans a row-tile boundary gets fewer pairs, and no range starts a row tile it cannot spend at least one pair on.  The
-// smallest per-range cost limit that needs no more than `resident` ranges is found by bisection; bound[] receives the
-// range starts (bound[grid] = n_pairs).  Returns the number of ranges.  Plans are cached per thread.
-int plan_ranges(int n_rt, int n_cs, int K, int NH, int resident, int* bound) {
-    struct Plan { int n_rt, n_cs, K, NH, resident, grid; int bound[kMaxGrid + 1]; };
-    static thread_local std::vector<Plan> plans;
-    for (const Plan& pl : plans)
-        if (pl.n_rt == n_rt && pl.n_cs == n_cs && pl.K == K && pl.NH == NH && pl.resident == resident) {
-            std::memcpy(bound, pl.bound, sizeof(pl.bound));
-            return pl.grid;
-        }
-    // fitted to timelines on B200: a pair is 8 K tiles at about 0.07 (NH = 1) or 0.085 us (NH = 2) each per CTA, a segment end 3 to 4 us
-    const double seg = (NH == 1 ? 3.0 : 4.0) / (8.0 * K * (NH == 1 ? 0.07 : 0.085));
+// Cuts the n_rt * n_cs (row tile, slice) pairs, in that order, into one contiguous range per SM, all the same length to
+// within one pair, and every SM's range into two parts, one per group of its CTA.  What has to be equal is the work of an
+// SM, not of a group: while one group adds up a segment and waits for its atomics, the other has the SM to itself, so a
+// group whose part spans a row-tile boundary (two segments) costs its SM next to nothing, whereas two long parts on one
+// SM and two short ones on the next (what equal-cost parts handed to independent CTAs gave, two per SM wherever the
+// hardware put them) made the launch wait for the slowest SM.  The cut between the two parts sits in the middle of the
+// SM's range, or on a row-tile boundary if one lies within a quarter of the range's length of the middle (one segment
+// fewer).  bound[] receives the starts of the 2 * grid parts (bound[2 * grid] = n_pairs); returns grid.
+int plan_ranges(int n_rt, int n_cs, int sms, int* bound) {
     const long long n_pairs = (long long)n_rt * n_cs;
-    auto cut = [&](double limit, int* out) {                             // greedy walk; returns the number of ranges (may exceed resident: then out is not filled further)
-        int n = 0;
-        long long u = 0;
-        while (u < n_pairs) {
-            if (n < resident && out) out[n] = (int)u;
-            ++n;
-            if (n > resident && !out) return n;
-            double c = 0.0;
-            bool first = true;
-            while (u < n_pairs) {
-                const long long left = n_cs - u % n_cs;                  // pairs to the end of this row tile
-                long long take = (long long)(limit - c - seg);           // pairs the budget still pays for after the segment's end
-                if (take < 1) {
-                    if (!first) break;                                   // do not start a segment the range cannot use
-                    take = 1;
-                }
-                if (take > left) take = left;
-                u += take;
-                c += seg + (double)take;
-                first = false;
-            }
-        }
-        return n;
-    };
-    double lo = seg + 1.0, hi = seg * (n_rt + 1) + (double)n_pairs + 1.0;
-    if (cut(lo, nullptr) > resident) {
-        for (int it = 0; it < 48; ++it) {
-            const double mid = 0.5 * (lo + hi);
-            if (cut(mid, nullptr) <= resident) hi = mid; else lo = mid;
-        }
-    } else {
-        hi = lo;
+    const int grid = (int)std::min<long long>(std::min(sms, kMaxRanges / kGroups), n_pairs);
+    for (int c = 0; c < grid; ++c) {
+        const long long a = n_pairs * c / grid, b = n_pairs * (c + 1) / grid, len = b - a;
+        long long mid = a + (len + 1) / 2;
+        const long long t = (a / n_cs + 1) * n_cs;                       // first row-tile boundary after a
+        const long long slack = std::max<long long>(1, len / 4);
+        if (t > a && t < b && t - mid <= slack && mid - t <= slack) mid = t;
+        bound[kGroups * c] = (int)a;
+        bound[kGroups * c + 1] = (int)mid;
     }
-    int tmp[kMaxGrid + 1];
-    const int grid = cut(hi, tmp);
-    for (int c = 0; c <= kMaxGrid; ++c) bound[c] = c < grid ? tmp[c] : (int)n_pairs;
-    if (plans.size() >= 256) plans.clear();
-    plans.emplace_back();
-    Plan& pl = plans.back();
-    pl.n_rt = n_rt; pl.n_cs = n_cs; pl.K = K; pl.NH = NH; pl.resident = resident; pl.grid = grid;
-    std::memcpy(pl.bound, bound, sizeof(pl.bound));
+    for (int r = kGroups * grid; r <= kMaxRanges; ++r) bound[r] = (int)n_pairs;
     return grid;
 }
 
@@ -440,7 +416,6 @@ cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, 
     P.two_pow_8 = 256u;
     P.n_pairs = G.n_rt * G.n_cs;
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
-    const int resident = std::min(2 * sms, kMaxGrid);                    // two CTAs per SM
-    const int grid = plan_ranges(G.n_rt, G.n_cs, G.K, batch > 8 ? 2 : 1, resident, P.bound);
+    const int grid = plan_ranges(G.n_rt, G.n_cs, sms, P.bound);       // one CTA (two groups of eight warps) per SM
     return batch <= 8 ? launch<1>(P, grid, L.device, stream) : launch<2>(P, grid, L.device, stream);
 }
