@@ -484,7 +484,7 @@ def bench_extras(args, rabit, device, stream, shapes, layers, peaks) -> dict:
                                             "note": "one token = one CUDA graph of %d launches (plus three tiny launches that select the token's "
                                                     "activations by a device-side index); tokens/s = 256 / elapsed" % (len(layers) * len(GROUPS))}
 
-    # config 3 / 4 samples at batch 1, batches 1, 8 and 16 on the 8B shapes, the batch-512 GEMM, and K = 1 / 3 at 7B shapes
+    # config 3 / 4 samples at batch 1, batches 1, 2, 4, 8 and 16 on the 8B shapes, the batch-512 GEMM, and K = 1 / 3 at 7B shapes
     extra_hbm = []
     for (M, N) in [(14336, 4096), (28672, 8192)]:
         lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 4)
@@ -505,14 +505,14 @@ def bench_extras(args, rabit, device, stream, shapes, layers, peaks) -> dict:
     b16 = []
     for (M, N) in [(4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336)]:
         lys = make_copies(M, N, K_PATHS, n_copies(M, N, K_PATHS), 3)
-        for batch in (1, 8, 16):
+        for batch in (1, 2, 4, 8, 16):
             x = torch.from_numpy(make_x(batch, N, key=(3, batch, N))).to(device)
             y = torch.zeros((batch, M), dtype=torch.float16, device=device)
             b16.append(hbm_case(M, N, K_PATHS, batch, timed_case(lys, x, y)))
         for L in lys:
             L.free()
         del lys
-    out["llama3_8b_shapes_batch_1_8_16"] = b16
+    out["llama3_8b_shapes_batch_1_to_16"] = b16
     kk = []
     for K in (1, 3):
         for (M, N) in [(4096, 4096), (11008, 4096)]:
@@ -690,7 +690,7 @@ def bench_cases(args) -> dict:
             "value": head["tflops"] if gemm else head["us_per_layer"], "unit": "TFLOP/s" if gemm else UNIT,
             "n_gpus": 1, "steps": args.steps, "warmup": 3, "ms_per_step": head["us_per_layer"] / 1e3,
             "higher_is_better": gemm, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f16 tensor-core products, fp32 accumulate" if gemm else "int8 tensor-core products of exact fixed-point activations",
+            "dtype": "f16 tensor-core products, fp32 accumulate" if gemm else "fp32 table sums (batch 1-2), f16 tensor-core products with fp32 accumulate (batch 3-16); 64-bit fixed-point cross-CTA sums",
             "data": "synthetic", "config": {"workload": args.workload, "K": K_PATHS,
                                             "l2": "rotation over distinct copies of each layer, > 4 x L2 in total where the layer is small"},
             "cases": cases, "roofline": head["roofline"], "clocks": clocks,
