@@ -118,7 +118,7 @@ def test_config3_llama3_8b_batch_sweep_sampled(batch):
         x = torch.from_numpy(xn).cuda()
         y = torch.zeros((batch, sh.M), dtype=torch.float16, device="cuda")
         _run_graph([layer], [x], [y])
-        if batch == 1:
+        if batch in (1, 16):                    # the table-driven kernel and the widest launch of the f16 GEMV: every row
             _check_all(L, xn, y.cpu().numpy())
         else:
             _check_rows(L, xn, y.cpu().numpy(), _sample_rows(sh.M, 32, seed=batch))
@@ -158,14 +158,14 @@ def _probe_columns(N, n_random=6, seed=0):
 def test_structured_probes_at_full_size(M, N):
     """Unit vectors and constant planes where a CTA owns many blocks, crosses slice borders and (tensor-core GEMV) wraps its
     ring: x = e_j reads exactly column j of the sign planes, so every row's output is one entry g*B*h of the weight and any
-    block that is skipped, repeated or attributed to the wrong rows or columns shows in some probe.  Batch 1, 2 and 4 (the
-    three decode launch shapes), every row compared under both bounds."""
+    block that is skipped, repeated or attributed to the wrong rows or columns shows in some probe.  Batch 1 and 2 (table-driven
+    kernel), 4, 8 and 16 (f16 tensor-core GEMV, one and two MMAs per operand), every row compared under both bounds."""
     import torch
     import paper_2602_05367_b200 as rabit
     L = make_layer(M, N, 2, key=(6, M, N))
     layer = rabit.rabit_pack(L.planes, L.g, L.h)
     cols = _probe_columns(N, seed=M)
-    for batch in (1, 2, 4):
+    for batch in (1, 2, 4, 8, 16):
         for c0 in range(0, len(cols), batch):
             js = cols[c0:c0 + batch]
             if len(js) < batch:
@@ -183,12 +183,13 @@ def test_structured_probes_at_full_size(M, N):
     for bit in (0, 1):
         planes = make_planes_constant(2, M, N, bit)
         layer = rabit.rabit_pack(planes, L.g, L.h)
-        xn = make_x(2, N, key=(6, bit, N))
-        y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
-        torch.cuda.synchronize()
-        dots = xn.astype(np.float64) @ L.h.astype(np.float64).T                       # [batch][K]
-        ref = (1.0 - 2.0 * bit) * dots @ L.g.astype(np.float64)                       # [batch][M]
-        compare(y.cpu().numpy().astype(np.float64), ref, orc.l1_bound(L.g, L.h, xn), orc.tolerance(L.g, L.h, xn))
+        for batch in (2, 16):
+            xn = make_x(batch, N, key=(6, bit, N, batch))
+            y = rabit.rabit_linear(layer, torch.from_numpy(xn).cuda())
+            torch.cuda.synchronize()
+            dots = xn.astype(np.float64) @ L.h.astype(np.float64).T                   # [batch][K]
+            ref = (1.0 - 2.0 * bit) * dots @ L.g.astype(np.float64)                   # [batch][M]
+            compare(y.cpu().numpy().astype(np.float64), ref, orc.l1_bound(L.g, L.h, xn), orc.tolerance(L.g, L.h, xn))
         layer.free()
 
 
