@@ -286,11 +286,13 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
         const int grp = e >> 2;
         // Exact form: warp e takes the words of packed lanes gq = e; its lanes spread over both column tiles, the two column
         // halves, the four tq and the two row halves, so that one 8-byte store per lane covers two whole 128-byte rows of
-        // the swizzled tile (all 32 banks twice, no conflict).
+        // the swizzled tile.  An 8-byte store is served half a warp at a time: lanes 0..15 must fill ONE row (16 x 8 bytes,
+        // all 32 banks once), so the row half is chosen by lane bit 4 and the position in the row by bits 0..3 (with the
+        // row half in bit 0 every half warp wrote two half rows on the same banks: 25 M of 42 M wavefronts were conflicts).
         // Dequantised form: a group has four warps, so warp e & 3 takes gq = 2*(e & 3) and 2*(e & 3) + 1 in turn.
-        const int x_ct2 = lane >> 4;
-        const int x_a = 2 * ((lane >> 3) & 1) + (lane & 1);
-        const int x_tq = (lane >> 1) & 3;
+        const int x_ct2 = (lane >> 3) & 1;
+        const int x_a = 2 * ((lane >> 2) & 1) + (lane >> 4);
+        const int x_tq = lane & 3;
         const int x_gq = DEQ ? 2 * (e & 3) : e;
         const int x_l = 4 * x_gq + x_tq;
         const int x_hoff = 32 * x_ct2 + 16 * (x_a >> 1) + 4 * x_tq;
