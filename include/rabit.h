@@ -85,7 +85,7 @@ RABIT_API int rabit_unpack_host(const void* image, size_t image_bytes,
  *   stream    the copy is enqueued on it and the call returns after it has completed.
  *   out       receives the new descriptor.
  * dev_buf also holds the layer's reduction scratch, in its resting state: the fp32 exchange buffer of the tensor-core
- * GEMV is all-ones words (0xFFFFFFFF, "nothing published"), the 64-bit accumulate words of the table-driven GEMV, the
+ * GEMV is all-ones words (0xFFFFFFFF, "nothing published"), the 64-bit accumulate words of the table-driven and f16 GEMVs, the
  * reserved flags and the status word are zero.  Every call leaves it in that state, so calls on one layer must not
  * overlap in time (different layers may).  A caller that moves or restores an image must keep these values.
  */
