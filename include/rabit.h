@@ -117,7 +117,7 @@ RABIT_API int rabit_derive_pack(const float* W_dev, const uint16_t* g, const uin
  * a CUDA graph.  The layer's device must be the current device.  One or two batch rows run the table-driven
  * GEMV (one pass over the weights: a shared-memory table of the partial sums of h*x over eight columns, indexed by the
  * packed sign byte), 3 to 16 rows the f16 tensor-core GEMV (one pass: the signs are expanded to +-h operand tiles in
- * registers, the batch is the MMA's N dimension), more than 16 the tcgen05 GEMM.  Layers those two GEMVs cannot take
+ * registers, the batch is the MMA's N dimension), 17 to 32 rows two passes of it, more the tcgen05 GEMM.  Layers those two GEMVs cannot take
  * (more than 255 slices of 256 input columns) fall back to the integer tensor-core GEMV, four rows per pass, or to one
  * GEMM launch, whichever the library's cost estimate for the shape favours.  A GEMM with few output tiles runs as
  * clusters of CTAs that share a tile's contraction.  fp32 (or exact integer) accumulation, one rounding to fp16 at the end;
@@ -266,7 +266,7 @@ RABIT_API int rabit_layer_N(const rabit_layer* layer);
  *   4 = tcgen05 GEMM on the dequantised weight tile sum_k +-g_k h_k rounded to fp16 (Eq. 2 formed per tile; one
  *       contraction of length N instead of K of them; never chosen automatically: it rounds every weight to fp16),
  *   5 = table-driven GEMV (passes of up to two batch rows; N up to 65280),
- *   6 = f16 tensor-core GEMV (one pass for up to 16 batch rows; N up to 65280).
+ *   6 = f16 tensor-core GEMV (passes of up to 16 batch rows; N up to 65280).
  * Returns RABIT_INVALID_ARG for a variant that cannot run the layer.
  * Meant for A/B timing and profiling; results are within tolerance for every variant.
  */

@@ -166,8 +166,9 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
         const double packed_mb = (double)G.K * G.Mp * G.N / 8.0e6;
         if (rabit_gemv_lut_supports(*layer, batch)) {
             variant = 5;
-        } else if (rabit_gemv_f16_supports(*layer, batch)) {
-            variant = 6;                    // 3..16 rows: one pass over the weights with the batch in the MMA's N dimension
+        } else if (batch <= 2 * RABIT_MAX_GEMV_BATCH && rabit_gemv_f16_supports(*layer, RABIT_MAX_GEMV_BATCH)) {
+            variant = 6;                    // 3..16 rows: one pass over the weights with the batch in the MMA's N dimension;
+                                            // 17..32: two passes, which measured faster than one GEMM launch on every shape tried
         } else if (batch <= 4 && packed_mb <= 8.0 && rabit_gemv_lut_supports(*layer, 1)) {
             variant = 5;                    // two passes of the table-driven kernel
         } else if (batch <= RABIT_MAX_GEMV_BATCH) {
@@ -216,9 +217,12 @@ extern "C" int rabit_linear(const rabit_layer* layer, const void* x, void* y, in
             break;
         }
         case 6:
-            if (!rabit_gemv_f16_supports(*layer, batch))
-                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: f16 tensor-core GEMV cannot run batch %d", batch);
-            e = rabit_launch_gemv_f16(*layer, x, y, batch, st);
+            if (!rabit_gemv_f16_supports(*layer, batch < RABIT_MAX_GEMV_BATCH ? batch : RABIT_MAX_GEMV_BATCH))
+                return rabit_fail(RABIT_INVALID_ARG, "rabit_linear: f16 tensor-core GEMV cannot run this layer");
+            e = cudaSuccess;
+            for (int b0 = 0; b0 < batch && e == cudaSuccess; b0 += RABIT_MAX_GEMV_BATCH)   // up to 16 batch rows share one pass over the weights
+                e = rabit_launch_gemv_f16(*layer, (const char*)x + (size_t)b0 * G.N * 2, (char*)y + (size_t)b0 * G.M * 2,
+                                          batch - b0 >= RABIT_MAX_GEMV_BATCH ? RABIT_MAX_GEMV_BATCH : batch - b0, st);
             break;
         default:
             e = rabit_launch_plain(*layer, x, y, batch, st);

@@ -75,15 +75,15 @@ def test_gemm_runs_small_batches_too(K, M, N, batch):
     check_against_oracle(L, x, y)
 
 
-@pytest.mark.parametrize("batch", [2, 3, 4, 8, 12, 16, 17])
+@pytest.mark.parametrize("batch", [2, 3, 4, 8, 12, 16, 17, 32, 33])
 def test_dispatch_by_batch(batch):
-    """One or two rows take the table-driven GEMV, 3 to 16 the f16 tensor-core GEMV, more the GEMM.  Whichever kernel
-    runs, the result is within tolerance and is exactly what that kernel gives when forced."""
+    """One or two rows take the table-driven GEMV, 3 to 32 the f16 tensor-core GEMV (passes of 16 rows), more the GEMM.
+    Whichever kernel runs, the result is within tolerance and is exactly what that kernel gives when forced."""
     L = make_layer(14336, 512, 2, key=(63,))
     x = make_x(batch, 512, key=(63, batch))
     y_auto = run_layer(L, x, 0)
     check_against_oracle(L, x, y_auto)
-    expect = 5 if batch <= 2 else 6 if batch <= 16 else GEMM
+    expect = 5 if batch <= 2 else 6 if batch <= 32 else GEMM
     y_forced = run_layer(L, x, expect)
     assert np.array_equal(y_auto.view(np.uint16), y_forced.view(np.uint16))
 
