@@ -396,6 +396,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
 #pragma unroll 1
             for (int c0 = 0; c0 < kTileB / 2; c0 += 32) {
                 const int col = col_half * (kTileB / 2) + c0;
+                if (bt * kTileB + col >= P.batch) break;                          // batch rows beyond the batch: nothing to drain or store
                 float v[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) v[c] = 0.f;
@@ -446,6 +447,7 @@ rabit_gemm_tc_kernel(const GemmParams P, const __grid_constant__ CUtensorMap x_m
 #pragma unroll 1
             for (int c0 = 0; c0 < kTileB / 2; c0 += 32) {
                 const int col = col_half * (kTileB / 2) + c0;
+                if (bt * kTileB + col >= P.batch) break;                          // batch rows beyond the batch: nothing to drain or store
                 float v[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) v[c] = 0.f;
