@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librabit.so")
 LIB_TRACE = os.path.join(HERE, "librabit_trace.so")          # the same sources with -DRABIT_TRACE (phase stamps)
-LIB_CHECKED = os.path.join(HERE, "librabit_checked.so")      # the same sources with -DRABIT_CHECKED (index checks in the decode kernel)
+LIB_CHECKED = os.path.join(HERE, "librabit_checked.so")      # the same sources with -DRABIT_CHECKED (index checks in the decode kernels)
 SOURCES = ["rabit_api.cu", "rabit_pack.cu", "rabit_gemv_plain.cu", "rabit_gemv_mma.cu", "rabit_gemv_lut.cu", "rabit_gemv_f16.cu", "rabit_gemm_tc.cu",
            "rabit_noalloc.cu", "rabit_derive.cu", "rabit_selftest.cu"]
 NVCC_FLAGS = [

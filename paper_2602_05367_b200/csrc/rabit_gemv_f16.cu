@@ -66,6 +66,7 @@ struct F16Params {
     const __half* x;
     __half* y;
     unsigned long long* acc;        // [16][Mp], all zero between calls
+    unsigned int* status;           // RABIT_CHECKED builds: set to 2 when an index check fails (the access is skipped)
     int K, M, N, Mp, n_rt, n_ct, n_cs;
     int batch;
     int n_pairs;                    // n_rt * n_cs (row tile, slice) pairs; group q of CTA c owns pairs [bound[2c + q], bound[2c + q + 1])
@@ -74,6 +75,15 @@ struct F16Params {
     uint32_t two, two_pow_8;        // 2 and 256: multipliers the compiler cannot fold into shifts
     int bound[kMaxRanges + 1];      // ascending; bound[2 * grid] = n_pairs
 };
+
+// Checked build (-DRABIT_CHECKED, python paper_2602_05367_b200/build.py --checked): every index that addresses global or
+// shared memory is compared with its range first; a violation is recorded in the layer's status word and the access is
+// skipped (nothing traps).  In the ordinary build the checks compile to nothing.
+#ifdef RABIT_CHECKED
+#define RABIT_IN_RANGE(cond) ((cond) ? true : (atomicExch(P.status, 2u), false))
+#else
+#define RABIT_IN_RANGE(cond) true
+#endif
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
     uint32_t r;
@@ -192,7 +202,10 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
     };
     auto prefill = [&](const Segment& sg) {                              // the first kRing - 1 tiles of the warp; weights never depend on the stream's past
 #pragma unroll
-        for (int i = 0; i < kRing - 1; ++i) copy_async_16(ring + i * 512, sg.wsrc + (size_t)i * n_same * 32, i < sg.n_my);
+        for (int i = 0; i < kRing - 1; ++i)
+            copy_async_16(ring + i * 512, sg.wsrc + (size_t)i * n_same * 32,
+                          i < sg.n_my && RABIT_IN_RANGE(sg.wsrc + (size_t)i * n_same * 32 >= P.tiles &&
+                                                        sg.wsrc + (size_t)i * n_same * 32 < P.tiles + (size_t)P.n_rt * P.K * P.n_ct * 32));
     };
     bool more = u < u_end;
     Segment sg;
@@ -214,9 +227,11 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
         // input scales and activations of the lane's four columns of k-step kh of column tile ct, as loaded (columns 0,1 | 2,3)
         auto fetch_hx = [&](int ct, int kh, uint2& fh, uint2 (&fx)[NH]) {
             const int off = ct * 32 + 16 * kh;
+            if (!RABIT_IN_RANGE(off >= 0 && hk + off + 4 <= P.K * P.N)) return;
             fh = __ldg(reinterpret_cast<const uint2*>(P.h + hk + off));
 #pragma unroll
-            for (int hf = 0; hf < NH; ++hf) fx[hf] = __ldcg(reinterpret_cast<const uint2*>(P.x + xb[hf] + off));
+            for (int hf = 0; hf < NH; ++hf)
+                if (RABIT_IN_RANGE(xb[hf] + off + 4 <= P.batch * P.N)) fx[hf] = __ldcg(reinterpret_cast<const uint2*>(P.x + xb[hf] + off));
         };
 
         // weights kRing - 1 tiles ahead (HBM latency), scales and activations one tile ahead, k-step by k-step in place
@@ -231,7 +246,9 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             {
                 const int ct = ct0 + i * n_same;
                 const int ia = i + kRing - 1;                            // the tile that takes the slot freed in the last round
-                copy_async_16(ring + (ia & (kRing - 1)) * 512, wsrc + (size_t)ia * n_same * 32, ia < n_my);
+                copy_async_16(ring + (ia & (kRing - 1)) * 512, wsrc + (size_t)ia * n_same * 32,
+                              ia < n_my && RABIT_IN_RANGE(wsrc + (size_t)ia * n_same * 32 >= P.tiles &&
+                                                          wsrc + (size_t)ia * n_same * 32 < P.tiles + (size_t)P.n_rt * P.K * P.n_ct * 32));
                 copy_async_wait<kRing - 1>();                            // tile i has landed (one group per tile, also for the tiles that do not exist)
                 const uint4 wv = lds_128(ring + (i & (kRing - 1)) * 512);
                 const int ct_next = min(ct + n_same, P.n_ct - 1);        // beyond the segment: a valid address, never used
@@ -277,10 +294,12 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             gk[kk] = kk < P.K ? P.g[(size_t)kk * P.Mp + rt * RABIT_TILE_ROWS + (tid & 127)] : __half();
         // ---- the warp's partial outputs -> its slot; slot layout [batch row][row of the tile]
         float* mine = slots + (size_t)warp * (NH * 8 * kSlotStride);
+        const bool slot_ok = RABIT_IN_RANGE(mine + (NH * 8 - 1) * kSlotStride + 127 < smem_f + kGroups * kGroupFloats);
 #pragma unroll
         for (int p = 0; p < 8; ++p)
 #pragma unroll
             for (int hf = 0; hf < NH; ++hf) {
+                if (!slot_ok) break;
                 const int b = 8 * hf + 2 * tq, row = 16 * p + gq;
                 mine[(b) * kSlotStride + row] = acc[p][hf][0];
                 mine[(b + 1) * kSlotStride + row] = acc[p][hf][1];
@@ -314,6 +333,7 @@ rabit_gemv_f16_kernel(const __grid_constant__ F16Params P) {
             old[i] = 0ULL;
             if (b >= P.batch) continue;
             unsigned long long* word = P.acc + (size_t)b * P.Mp + rt * RABIT_TILE_ROWS + rl;
+            if (!RABIT_IN_RANGE(rt * RABIT_TILE_ROWS + rl < P.Mp && b < RABIT_LUT_MAX_BATCH)) continue;
             if (bad[i]) atomicOr(word, 1ULL << 63);                      // sticky: the add below never carries into bit 63
             old[i] = atomicAdd(word, add[i]);
         }
@@ -406,6 +426,7 @@ cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, 
     P.x = (const __half*)x;
     P.y = (__half*)y;
     P.acc = L.d_acc;
+    P.status = L.d_status;
     P.K = G.K; P.M = G.M; P.N = G.N; P.Mp = G.Mp; P.n_rt = G.n_rt; P.n_ct = G.n_ct; P.n_cs = G.n_cs;
     P.batch = batch;
     P.fix_bits = G.fix_bits;

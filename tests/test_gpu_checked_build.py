@@ -1,5 +1,5 @@
 """The small-shape parity suite under the checked build of the library (-DRABIT_CHECKED): every index that addresses
-memory in the table-driven decode kernel is compared with its range first, a violation sets the layer's status word and
+memory in the decode kernels (table-driven and f16 GEMV) is compared with its range first, a violation sets the layer's status word and
 skips the access.  This stands in for a memory checker: the suite must pass with a clear status word.  The checked library
 is a separate file (librabit_checked.so) selected through RABIT_LIBRARY, so it runs in a child process."""
 import importlib.util
