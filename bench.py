@@ -743,7 +743,7 @@ def bench_derive(args) -> dict:
         cases.append({"M": sh.M, "N": sh.N, "us": us, "gbs": nbytes / us / 1e3,
                       "roofline": {"bound": "hbm", "achieved": nbytes / us / 1e3, "peak": hbm_peak, "unit": "GB/s", "frac": nbytes / us / 1e3 / hbm_peak},
                       "note": "back-to-back asynchronous calls through the C ABI, CUDA events around all of them: includes the "
-                              "upload of header and scales and two fills per call"})
+                              "upload of the scales, the second kernel (look-up blocks, scratch fills, header) and the fill of the accumulate words"})
         del Ws
         torch.cuda.empty_cache()
     head = max(cases, key=lambda c: c["M"] * c["N"])

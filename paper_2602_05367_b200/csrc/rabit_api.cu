@@ -115,14 +115,15 @@ extern "C" int rabit_derive_pack(const float* W_dev, const uint16_t* g, const ui
         return rabit_fail(RABIT_INVALID_ARG, "rabit_derive_pack: W overlaps dev_buf");
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)dev_buf;
-    RABIT_CUDA_TRY(cudaMemcpyAsync(base, &hdr, sizeof(hdr), cudaMemcpyHostToDevice, st));
-    // scales from the host (a few KB), the scratch sections by device-side fills
+    // scales from the host (a few KB); the header travels as a parameter of the second kernel
     RABIT_CUDA_TRY(cudaMemcpyAsync(base + hdr.off_g, tail.data(), tail.size(), cudaMemcpyHostToDevice, st));
-    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_partial, 0xFF, (size_t)(hdr.off_flags - hdr.off_partial), st));
-    RABIT_CUDA_TRY(cudaMemsetAsync(base + hdr.off_flags, 0, (size_t)(hdr.off_lut - hdr.off_flags), st));
     cudaError_t e = rabit_launch_derive(G, W_dev, (const uint16_t*)(base + hdr.off_g), (const uint16_t*)(base + hdr.off_h),
                                         (uint4*)(base + hdr.off_bits), st);
-    if (e == cudaSuccess) e = rabit_launch_tiles_to_lut(G, (const uint4*)(base + hdr.off_bits), (unsigned char*)(base + hdr.off_lut), st);
+    // the second kernel also puts the exchange buffer (all-ones words) and the flags (zero) into their resting state
+    if (e == cudaSuccess)
+        e = rabit_launch_tiles_to_lut(G, (const uint4*)(base + hdr.off_bits), (unsigned char*)(base + hdr.off_lut),
+                                      base + hdr.off_partial, (size_t)(hdr.off_flags - hdr.off_partial),
+                                      base + hdr.off_flags, (size_t)(hdr.off_lut - hdr.off_flags), &hdr, base, st);
     if (e != cudaSuccess) return rabit_fail(RABIT_CUDA_ERROR, "rabit_derive_pack: launch failed: %s", cudaGetErrorString(e));
     // The accumulate words are cleared AFTER the kernels on purpose: the decode kernels start copying weights before
     // they wait for the previous kernel in the stream (weights normally never depend on it).  A fill between the

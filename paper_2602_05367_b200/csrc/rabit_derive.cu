@@ -9,6 +9,8 @@
 // exact in fp32, so each residual update is one fp32 rounding; sign(0) = +1 (bit 0).
 #include <cuda_fp16.h>
 
+#include <cstring>
+
 #include "rabit_internal.h"
 
 namespace {
@@ -83,52 +85,71 @@ rabit_derive_kernel(RabitGeom G, const float* __restrict__ W, const __half* __re
 }
 
 // Second arrangement of the same signs: the look-up blocks (rabit_layout.h), gathered from the tiles that the
-// kernel above has just written.  One warp per (path, row block of 32 rows, slice of 256 columns) = one 1 KB part;
-// lane = row.  A byte of eight consecutive columns comes from two tile words (four columns each, the row's bit p
-// in every byte).  Columns beyond N stay zero.
+// kernel above has just written.  One CTA per (row tile, slice of 256 columns): its eight warps first copy the slice's
+// 8 K sign tiles into shared memory (coalesced, every tile read once), then each warp gathers parts of 1 KB
+// (path k, row block of 32 rows; lane = row).  A byte of eight consecutive columns comes from two tile words (four
+// columns each, the row's bit p in every byte).  Columns beyond N stay zero.  The CTAs also share out two fills that put
+// the layer's reduction scratch into its resting state: `n_ones` 16-byte units of all-ones words, `n_zero` of zeros; and
+// the first CTA writes the image's header, which arrives as a kernel parameter (one host-to-device copy fewer).
+struct HeaderWords {
+    uint4 v[RABIT_HEADER_BYTES / 16];
+};
 __global__ void __launch_bounds__(kWarps * 32)
-rabit_tiles_to_lut_kernel(RabitGeom G, const uint32_t* __restrict__ tiles, uint4* __restrict__ lut) {
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
-    const long long parts = (long long)G.n_cs * G.n_rb * G.K;
-    if (wid >= parts) return;
-    const int k = (int)(wid % G.K);
-    const long long pos = wid / G.K;
-    const int rb = (int)(pos % G.n_rb), cs = (int)(pos / G.n_rb);
-    const int row = rb * RABIT_LUT_ROWS + lane;
-    const int rt = row >> 7, rl = row & 127, p = rl >> 4, gq = rl & 7, alo = (rl >> 3) & 1;
-    uint32_t out[8];
+rabit_tiles_to_lut_kernel(RabitGeom G, const uint4* __restrict__ tiles, uint4* __restrict__ lut,
+                          uint4* __restrict__ ones, size_t n_ones, uint4* __restrict__ zero, size_t n_zero,
+                          const __grid_constant__ HeaderWords header, uint4* __restrict__ header_dst) {
+    __shared__ uint4 staged[RABIT_MAX_K][kWarps][32];     // [path][column tile of the slice][lane of the tile]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && header_dst != nullptr && threadIdx.x < RABIT_HEADER_BYTES / 16) header_dst[threadIdx.x] = header.v[threadIdx.x];
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_ones; i += (size_t)gridDim.x * blockDim.x)
+        ones[i] = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_zero; i += (size_t)gridDim.x * blockDim.x)
+        zero[i] = make_uint4(0u, 0u, 0u, 0u);
+    const int rt = blockIdx.x / G.n_cs, cs = blockIdx.x - rt * G.n_cs;
+    const int ct = cs * kWarps + warp;
+    for (int k = 0; k < G.K; ++k)
+        staged[k][warp][lane] = ct < G.n_ct ? tiles[rabit_tile_pos(G, rt, k, ct) * 32 + lane] : make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    for (int part = warp; part < 4 * G.K; part += kWarps) {
+        const int k = part % G.K, rbl = part / G.K;
+        const int rl = rbl * RABIT_LUT_ROWS + lane;                     // row inside the tile
+        const int p = rl >> 4, gq = rl & 7, alo = (rl >> 3) & 1;
+        uint32_t o[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) out[j] = 0u;
-#pragma unroll 4
-    for (int s = 0; s < 32; ++s) {
-        const int group = (s + lane) & 31;                              // byte group of the slice this lane stores at step s
-        const int col = cs * RABIT_LUT_COLS + 8 * group;
-        uint32_t byte = 0u;
-        if (col < G.N) {
-            const int ct = col >> 5, cl = col & 31, ah = cl >> 4, tq0 = (cl & 15) >> 2;     // tq0 is 0 or 2
-            const uint32_t* tile = tiles + rabit_tile_pos(G, rt, k, ct) * (RABIT_TILE_BYTES / 4);
-            const int a = alo | (ah << 1);
-            const uint32_t w0 = tile[(4 * gq + tq0) * 4 + a], w1 = tile[(4 * gq + tq0 + 1) * 4 + a];
+        for (int j = 0; j < 8; ++j) o[j] = 0u;
+#pragma unroll
+        for (int sidx = 0; sidx < 32; ++sidx) {
+            const int group = (sidx + lane) & 31;                       // byte group of the slice this lane stores at step sidx
+            const int ctl = group >> 2, ah = (group >> 1) & 1, tq0 = (group & 1) * 2;
+            const uint32_t* words = reinterpret_cast<const uint32_t*>(&staged[k][ctl][4 * gq + tq0]);
+            const uint32_t w0 = words[alo | (ah << 1)], w1 = words[4 + (alo | (ah << 1))];
             const uint32_t n0 = ((((w0 >> p) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;  // bit c <- byte c
             const uint32_t n1 = ((((w1 >> p) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;
-            byte = n0 | (n1 << 4);
+            o[sidx >> 2] |= (n0 | (n1 << 4)) << (8 * (sidx & 3));
         }
-        out[s >> 2] |= byte << (8 * (s & 3));
+        const int rb = rt * (RABIT_TILE_ROWS / RABIT_LUT_ROWS) + rbl;
+        uint4* dst = lut + (((size_t)cs * G.n_rb + rb) * G.K + k) * (RABIT_LUT_PART_BYTES / 16);
+        dst[lane] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[32 + lane] = make_uint4(o[4], o[5], o[6], o[7]);
     }
-    uint4* dst = lut + (size_t)wid * (RABIT_LUT_PART_BYTES / 16);
-    dst[lane] = make_uint4(out[0], out[1], out[2], out[3]);
-    dst[32 + lane] = make_uint4(out[4], out[5], out[6], out[7]);
 }
 
 }  // namespace
 
-cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, cudaStream_t stream) {
-    const long long warps = (long long)G.n_cs * G.n_rb * G.K;
-    const long long blocks = (warps + kWarps - 1) / kWarps;
+cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, void* d_ones, size_t ones_bytes,
+                                      void* d_zero, size_t zero_bytes, const RabitHeader* header, void* d_header, cudaStream_t stream) {
+    static_assert(sizeof(RabitHeader) == RABIT_HEADER_BYTES, "the header travels as a kernel parameter");
+    HeaderWords hw;
+    std::memset(&hw, 0, sizeof(hw));
+    if (header) std::memcpy(&hw, header, sizeof(RabitHeader));
+    if ((ones_bytes | zero_bytes | (size_t)(uintptr_t)d_ones | (size_t)(uintptr_t)d_zero) & 15u) return cudaErrorInvalidValue;
+    static_assert(kWarps * RABIT_TILE_COLS == RABIT_LUT_COLS, "one warp per column tile of a slice");
+    const long long blocks = (long long)G.n_rt * G.n_cs;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-    rabit_tiles_to_lut_kernel<<<(unsigned int)blocks, kWarps * 32, 0, stream>>>(G, reinterpret_cast<const uint32_t*>(d_tiles),
-                                                                               reinterpret_cast<uint4*>(d_lut));
+    rabit_tiles_to_lut_kernel<<<(unsigned int)blocks, kWarps * 32, 0, stream>>>(G, d_tiles, reinterpret_cast<uint4*>(d_lut),
+                                                                               reinterpret_cast<uint4*>(d_ones), ones_bytes / 16,
+                                                                               reinterpret_cast<uint4*>(d_zero), zero_bytes / 16, hw,
+                                                                               header ? reinterpret_cast<uint4*>(d_header) : nullptr);
     return cudaGetLastError();
 }
 

@@ -51,7 +51,10 @@ bool rabit_build_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N,
 cudaError_t rabit_launch_derive(const RabitGeom& G, const float* W, const uint16_t* d_g, const uint16_t* d_h, uint4* d_tiles,
                                 cudaStream_t stream);
 
-cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, cudaStream_t stream);
+// gathers the look-up blocks from the sign tiles, fills ones_bytes at d_ones with 0xFF and zero_bytes at d_zero with 0 (16-byte
+// units) and, if header is not null, writes it (256 bytes, passed as a kernel parameter) to d_header
+cudaError_t rabit_launch_tiles_to_lut(const RabitGeom& G, const uint4* d_tiles, unsigned char* d_lut, void* d_ones, size_t ones_bytes,
+                                      void* d_zero, size_t zero_bytes, const RabitHeader* header, void* d_header, cudaStream_t stream);
 
 // kernel launchers; each enqueues on `stream` and returns a cudaError_t from the launch
 cudaError_t rabit_launch_plain(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);

@@ -52,28 +52,43 @@ bool rabit_make_geom(int K, int M, int N, RabitGeom* out) {
 //     65504 * max_i sum_k |g_k[i]| * max_{k, slice} sum_{j in slice} |h_k[j]|,
 // so a grid of 2^unit_exp whose 2^fix_bits steps cover twice that bound can never overflow, and with
 // fix_bits = 54 - ceil(log2(slices)) the sum of all slices (each shifted to be non-negative) stays below 2^55.
+// |value| of every fp16 magnitude (sign bit cleared), converted once: the scans below are table look-ups
+static const float* half_magnitude_table() {
+    static const std::vector<float> table = [] {
+        std::vector<float> t(32768);
+        for (uint32_t m = 0; m < 32768; ++m) t[m] = half_bits_to_float((uint16_t)m);
+        return t;
+    }();
+    return table.data();
+}
+
 void rabit_scale_meta(const uint16_t* g, const uint16_t* h, int K, int M, int N, RabitGeom* G) {
+    const float* mag = half_magnitude_table();
+    // one pass over h: per path the largest |h| (fp16 magnitudes order like their bit patterns; the first NaN wins and
+    // sticks, so a NaN scale makes the bound NaN) and per slice of 256 columns the sum of |h|, added in column order
+    double hsum_max = 0.0;
     for (int k = 0; k < K; ++k) {
-        float m = 0.f;
-        for (int j = 0; j < N; ++j) {
-            const float v = std::fabs(half_bits_to_float(h[(size_t)k * N + j]));
-            if (m == m && (v > m || v != v)) m = v;   // a NaN scale makes the bound NaN
+        const uint16_t* hk = h + (size_t)k * N;
+        uint32_t top = 0, first_nan = 0;
+        for (int j0 = 0; j0 < N; j0 += RABIT_LUT_COLS) {
+            const int j1 = j0 + RABIT_LUT_COLS < N ? j0 + RABIT_LUT_COLS : N;
+            double s = 0.0;
+            for (int j = j0; j < j1; ++j) {
+                const uint32_t m = hk[j] & 0x7FFFu;
+                if (m > 0x7C00u && first_nan == 0) first_nan = m;
+                top = m > top ? m : top;
+                s += (double)mag[m];
+            }
+            if (s > hsum_max || s != s) hsum_max = s;
         }
-        G->hmax[k] = m;
+        G->hmax[k] = mag[first_nan ? first_nan : top];
     }
     double gsum_max = 0.0;
     for (int i = 0; i < M; ++i) {
         double s = 0.0;
-        for (int k = 0; k < K; ++k) s += std::fabs((double)half_bits_to_float(g[(size_t)k * M + i]));
+        for (int k = 0; k < K; ++k) s += (double)mag[g[(size_t)k * M + i] & 0x7FFFu];
         if (s > gsum_max || s != s) gsum_max = s;
     }
-    double hsum_max = 0.0;
-    for (int k = 0; k < K; ++k)
-        for (int j0 = 0; j0 < N; j0 += RABIT_LUT_COLS) {
-            double s = 0.0;
-            for (int j = j0; j < N && j < j0 + RABIT_LUT_COLS; ++j) s += std::fabs((double)half_bits_to_float(h[(size_t)k * N + j]));
-            if (s > hsum_max || s != s) hsum_max = s;
-        }
     int clog = 0;
     while ((1 << clog) < G->n_cs) ++clog;
     G->fix_bits = 54 - clog;
