@@ -51,6 +51,31 @@ def test_f16_tensor_core_gemv_batches(K, M, N, batch):
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))     # integer accumulate words: the same bits every run
 
 
+@pytest.mark.parametrize("batch", [1, 2, 5, 16])
+def test_widest_layer_of_the_accumulate_word_kernels(batch):
+    """N = 65280 is 255 slices of 256 columns, the most the eight-bit arrival count of an accumulate word can take: the
+    table-driven kernel (batch 1, 2) and the f16 GEMV (5, 16) at that limit, where a row's word collects up to 255
+    contributions on a grid of 46 magnitude bits."""
+    L = make_layer(200, 65280, 2, key=(70,))
+    x = make_x(batch, 65280, key=(70, batch))
+    y = run_layer(L, x, 0)
+    check_against_oracle(L, x, y)
+    forced = run_layer(L, x, 5 if batch <= 2 else 6)
+    assert np.array_equal(y.view(np.uint16), forced.view(np.uint16))
+
+
+def test_layer_wider_than_the_accumulate_word_kernels_falls_back():
+    """One more column tile (256 slices): both kernels refuse the layer, the dispatcher takes the integer-MMA GEMV or the GEMM."""
+    import paper_2602_05367_b200 as rabit
+    L = make_layer(200, 65312, 2, key=(71,))
+    for batch in (1, 5):
+        x = make_x(batch, 65312, key=(71, batch))
+        check_against_oracle(L, x, run_layer(L, x, 0))
+        for variant in (5, 6):
+            with pytest.raises(rabit.RabitError):
+                run_layer(L, x, variant)
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_config0_full_size(variant):
     """4096 x 4096, K=2, batch 1, seed 0 -- every output compared."""
