@@ -382,27 +382,84 @@ cudaError_t launch(const F16Params& P, int grid, int device, cudaStream_t stream
 
 namespace {
 
-// Cuts the n_rt * n_cs (row tile, slice) pairs, in that order, into one contiguous range per SM, all the same length to
-// within one pair, and every SM's range into two parts, one per group of its CTA.  What has to be equal is the work of an
-// SM, not of a group: while one group adds up a segment and waits for its atomics, the other has the SM to itself, so a
-// group whose part spans a row-tile boundary (two segments) costs its SM next to nothing, whereas two long parts on one
-// SM and two short ones on the next (what equal-cost parts handed to independent CTAs gave, two per SM wherever the
-// hardware put them) made the launch wait for the slowest SM.  The cut between the two parts sits in the middle of the
-// SM's range, or on a row-tile boundary if one lies within a quarter of the range's length of the middle (one segment
-// fewer).  bound[] receives the starts of the 2 * grid parts (bound[2 * grid] = n_pairs); returns grid.
-int plan_ranges(int n_rt, int n_cs, int sms, int* bound) {
+// Cuts the n_rt * n_cs (row tile, slice) pairs, in that order, into one contiguous range per SM and every SM's range into
+// two parts, one per group of its CTA.  A group's cost is its pairs plus `seg` for every segment after its first (a part
+// that crosses a row-tile boundary adds up and publishes twice, and while it does so its SM runs at half strength; the last
+// segment end is the same for everybody); an SM's cost is that of its slower group under the best cut between the two
+// parts, which is often the row-tile boundary itself.  The SM ranges are grown greedily under a cost limit and the
+// smallest limit that needs no more than `sms` ranges is found by bisection, so SMs whose range holds a boundary get
+// fewer pairs.  (Equal ranges cut in the middle, the previous form, left such SMs 30-40 % late; equal-cost parts
+// handed to independent CTAs, two per SM wherever the hardware put them, gave SMs unequal sums.)
+// bound[] receives the starts of the 2 * grid parts (bound[2 * grid] = n_pairs); returns grid.  Plans are cached per thread.
+int plan_ranges(int n_rt, int n_cs, int K, int NH, int sms, int* bound) {
+    struct Plan { int n_rt, n_cs, K, NH, sms, grid; int bound[kMaxRanges + 1]; };
+    static thread_local std::vector<Plan> plans;
+    for (const Plan& pl : plans)
+        if (pl.n_rt == n_rt && pl.n_cs == n_cs && pl.K == K && pl.NH == NH && pl.sms == sms) {
+            std::memcpy(bound, pl.bound, sizeof(pl.bound));
+            return pl.grid;
+        }
     const long long n_pairs = (long long)n_rt * n_cs;
-    const int grid = (int)std::min<long long>(std::min(sms, kMaxRanges / kGroups), n_pairs);
-    for (int c = 0; c < grid; ++c) {
-        const long long a = n_pairs * c / grid, b = n_pairs * (c + 1) / grid, len = b - a;
-        long long mid = a + (len + 1) / 2;
-        const long long t = (a / n_cs + 1) * n_cs;                       // first row-tile boundary after a
-        const long long slack = std::max<long long>(1, len / 4);
-        if (t > a && t < b && t - mid <= slack && mid - t <= slack) mid = t;
-        bound[kGroups * c] = (int)a;
-        bound[kGroups * c + 1] = (int)mid;
+    const int max_grid = (int)std::min<long long>(std::min(sms, kMaxRanges / kGroups), n_pairs);
+    // fitted to timelines on B200: a group works through a tile of a pair (8 K tiles) in about 0.068 us (NH = 1) or 0.085 us
+    // (NH = 2), a segment end takes it 3 to 3.5 us
+    const double seg = (NH == 1 ? 3.0 : 3.5) / (8.0 * K * (NH == 1 ? 0.068 : 0.085));
+    auto part_cost = [&](long long a, long long b) {                     // pairs [a, b) as one group's part
+        if (b <= a) return 0.0;
+        const long long segments = (b - 1) / n_cs - a / n_cs + 1;
+        return (double)(b - a) + seg * (double)(segments - 1);
+    };
+    auto best_cut = [&](long long a, long long b, double* cost) {        // the cut of [a, b) that makes the slower group fastest
+        long long best = b;
+        double best_cost = part_cost(a, b);
+        for (long long m = a + 1; m < b; ++m) {
+            const double c = std::max(part_cost(a, m), part_cost(m, b));
+            if (c < best_cost) { best_cost = c; best = m; }
+        }
+        *cost = best_cost;
+        return best;
+    };
+    auto cut_all = [&](double limit, int* out) {                         // greedy SM ranges under the limit; returns their number
+        int n = 0;
+        long long a = 0;
+        while (a < n_pairs) {
+            long long lo = a + 1, hi = std::min<long long>(n_pairs, a + 4 * (long long)limit + 8);   // largest b with cost <= limit
+            while (lo < hi) {
+                const long long mid = (lo + hi + 1) / 2;
+                double c;
+                best_cut(a, mid, &c);
+                if (c <= limit) lo = mid; else hi = mid - 1;
+            }
+            if (out && n < max_grid) {
+                double c;
+                out[kGroups * n] = (int)a;
+                out[kGroups * n + 1] = (int)best_cut(a, lo, &c);
+            }
+            ++n;
+            if (n > max_grid && !out) return n;
+            a = lo;
+        }
+        return n;
+    };
+    double lo = 1.0, hi = (double)n_pairs + seg * (n_rt + 1) + 1.0;
+    if (n_pairs <= max_grid) {
+        lo = hi = 0.5;                                                   // fewer pairs than SMs: one pair, one group per SM (a group alone on its SM is faster than two)
+    } else if (cut_all(lo, nullptr) > max_grid) {
+        for (int it = 0; it < 40; ++it) {
+            const double mid = 0.5 * (lo + hi);
+            if (cut_all(mid, nullptr) <= max_grid) hi = mid; else lo = mid;
+        }
+    } else {
+        hi = lo;
     }
-    for (int r = kGroups * grid; r <= kMaxRanges; ++r) bound[r] = (int)n_pairs;
+    int tmp[kMaxRanges + 2];
+    const int grid = cut_all(hi, tmp);
+    for (int r = 0; r <= kMaxRanges; ++r) bound[r] = r < kGroups * grid ? tmp[r] : (int)n_pairs;
+    if (plans.size() >= 256) plans.clear();
+    plans.emplace_back();
+    Plan& pl = plans.back();
+    pl.n_rt = n_rt; pl.n_cs = n_cs; pl.K = K; pl.NH = NH; pl.sms = sms; pl.grid = grid;
+    std::memcpy(pl.bound, bound, sizeof(pl.bound));
     return grid;
 }
 
@@ -437,6 +494,6 @@ cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, 
     P.two_pow_8 = 256u;
     P.n_pairs = G.n_rt * G.n_cs;
     const int sms = L.sm_count > 0 ? L.sm_count : 148;
-    const int grid = plan_ranges(G.n_rt, G.n_cs, sms, P.bound);       // one CTA (two groups of eight warps) per SM
+    const int grid = plan_ranges(G.n_rt, G.n_cs, G.K, batch > 8 ? 2 : 1, sms, P.bound);   // one CTA (two groups of eight warps) per SM
     return batch <= 8 ? launch<1>(P, grid, L.device, stream) : launch<2>(P, grid, L.device, stream);
 }
