@@ -24,7 +24,7 @@
 // and the accumulator lane holds rows gq, gq + 8 of the block and batch rows 2tq, 2tq + 1.
 //
 // Work split.  The layer is n_rt row tiles x n_cs slices of 256 columns; in that order the (row tile, slice) pairs are cut
-// into one contiguous range per SM, all the same length to within one pair, and every SM's range into two parts.  One
+// into one contiguous range per SM and every SM's range into two parts, by a cost model on the host (plan_ranges).  One
 // CTA of 16 warps per SM; its two groups of 8 warps each take one part and share nothing but the SM (own barrier, own
 // shared memory): while one group adds up a segment and waits for its atomics, the other computes.  The part of a range
 // inside one row tile is a segment.  Warp w of a group works on path w % K and shares the column tiles of the segment
