@@ -211,6 +211,15 @@ RABIT_API int rabit_layer_status(const rabit_layer* layer, int clear, void* stre
 RABIT_API int rabit_selftest_bounded_wait(unsigned int* status_dev, int limit_us, void* stream);
 
 /*
+ * Test aid (no counterpart in the paper; host only, no GPU needed): how the f16 tensor-core GEMV of rabit_linear
+ * (batch 3..16) would split a K-path layer of M x N at `batch` rows over `sms` SMs.  The layer is ceil(M/128) row tiles x
+ * ceil(N/256) slices; in that order the (row tile, slice) pairs are cut into contiguous parts, two per SM (one per group
+ * of eight warps).  bound_out (HOST, max_out ints) receives the starts of the parts followed by the number of pairs:
+ * 2 * grid + 1 ascending values; a part may be empty.  Returns the number of CTAs (grid >= 1), or RABIT_INVALID_ARG.
+ */
+RABIT_API int rabit_selftest_f16_plan(int K, int M, int N, int batch, int sms, int* bound_out, int max_out);
+
+/*
  * Measurement aid (no counterpart in the paper): one kernel that reads `bytes` bytes of device memory once with
  * 128-bit streaming loads and keeps nothing.  Timed by the caller with CUDA events over a buffer much larger than L2
  * it gives the read-only HBM bandwidth this GPU delivers to plain loads, the natural ceiling of the decode GEMV.

@@ -60,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.rabit_layer_status.argtypes = [_c_void_p, _c_int, _c_void_p]
     lib.rabit_selftest_bounded_wait.restype = _c_int
     lib.rabit_selftest_bounded_wait.argtypes = [_c_void_p, _c_int, _c_void_p]
+    lib.rabit_selftest_f16_plan.restype = _c_int
+    lib.rabit_selftest_f16_plan.argtypes = [_c_int, _c_int, _c_int, _c_int, _c_int, _c_void_p, _c_int]
     lib.rabit_selftest_stream_read.restype = _c_int
     lib.rabit_selftest_stream_read.argtypes = [_c_void_p, _c_size_t, _c_void_p, _c_void_p]
     lib.rabit_unpack.restype = _c_int

@@ -465,6 +465,19 @@ int plan_ranges(int n_rt, int n_cs, int K, int NH, int sms, int* bound) {
 
 }  // namespace
 
+// Host-only view of the work split (for tests): the starts of the 2 * grid group parts of a K-path layer of M x N at
+// `batch` rows on `sms` SMs; bound_out receives 2 * grid + 1 values, the last being the number of pairs.
+int rabit_gemv_f16_plan(int K, int M, int N, int batch, int sms, int* bound_out, int max_out) {
+    if (K < 1 || K > RABIT_MAX_K || M < 1 || N < 32 || (N % 32) != 0 || batch < 1 || batch > RABIT_MAX_GEMV_BATCH || sms < 1) return -1;
+    const long long n_rt = ((long long)M + RABIT_TILE_ROWS - 1) / RABIT_TILE_ROWS, n_cs = ((long long)N + RABIT_LUT_COLS - 1) / RABIT_LUT_COLS;
+    if (n_cs > RABIT_LUT_MAX_SLICES || n_rt * n_cs >= kMaxPairs) return -1;
+    int bound[kMaxRanges + 1];
+    const int grid = plan_ranges((int)n_rt, (int)n_cs, K, batch > 8 ? 2 : 1, sms, bound);
+    if (max_out < kGroups * grid + 1) return -1;
+    for (int r = 0; r <= kGroups * grid; ++r) bound_out[r] = bound[r];
+    return grid;
+}
+
 bool rabit_gemv_f16_supports(const rabit_layer& L, int batch) {
     if (batch < 1 || batch > RABIT_MAX_GEMV_BATCH) return false;
     if (L.geom.n_cs > RABIT_LUT_MAX_SLICES || L.d_acc == nullptr) return false;

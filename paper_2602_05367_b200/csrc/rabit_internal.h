@@ -74,6 +74,7 @@ unsigned long long* rabit_trace_slot(int ctas);
 // f16 tensor-core GEMV for 3..16 batch rows (rabit_gemv_f16.cu)
 cudaError_t rabit_launch_gemv_f16(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);
 bool rabit_gemv_f16_supports(const rabit_layer& L, int batch);
+int rabit_gemv_f16_plan(int K, int M, int N, int batch, int sms, int* bound_out, int max_out);   // host only: the work split
 
 // table-driven GEMV (rabit_gemv_lut.cu); acc_override / status_override redirect the scratch (nullptr: the image's own)
 cudaError_t rabit_launch_gemv_lut(const rabit_layer& L, const void* x, void* y, int batch, cudaStream_t stream);

@@ -48,6 +48,14 @@ __global__ void __launch_bounds__(512) stream_read_probe(const uint4* __restrict
 
 }  // namespace
 
+extern "C" int rabit_selftest_f16_plan(int K, int M, int N, int batch, int sms, int* bound_out, int max_out) {
+    rabit_clear_error();
+    if (!bound_out) return rabit_fail(RABIT_INVALID_ARG, "rabit_selftest_f16_plan: bound_out is NULL");
+    const int grid = rabit_gemv_f16_plan(K, M, N, batch, sms, bound_out, max_out);
+    if (grid < 0) return rabit_fail(RABIT_INVALID_ARG, "rabit_selftest_f16_plan: unsupported shape or too small an output array");
+    return grid;
+}
+
 extern "C" int rabit_selftest_stream_read(const void* src_dev, size_t bytes, unsigned int* sink_dev, void* stream) {
     rabit_clear_error();
     if (!src_dev || ((uintptr_t)src_dev & 15u)) return rabit_fail(RABIT_INVALID_ARG, "rabit_selftest_stream_read: src_dev must be a 16-byte aligned device pointer");

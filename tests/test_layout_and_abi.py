@@ -182,3 +182,51 @@ def test_every_declared_symbol_is_exported():
     lib = ctypes.CDLL(rabit.lib_path())
     for n in names:
         assert hasattr(lib, n), f"{n} declared in include/rabit.h but not exported"
+
+
+@pytest.mark.parametrize("K,M,N,batch,sms", [
+    (2, 14336, 4096, 16, 148), (2, 14336, 4096, 8, 148), (2, 4096, 4096, 16, 148), (2, 4096, 14336, 3, 148),
+    (2, 28672, 8192, 16, 148), (2, 1024, 4096, 8, 148), (3, 11008, 4096, 16, 148), (1, 129, 288, 5, 148),
+    (2, 200, 65280, 16, 148), (2, 128, 32, 3, 148), (2, 100000, 4096, 12, 148), (2, 4096, 11008, 16, 132), (2, 300, 640, 7, 4),
+])
+def test_work_split_of_the_f16_gemv(K, M, N, batch, sms):
+    """Host logic of the batch 3..16 kernel: the (row tile, slice) pairs are cut into two contiguous parts per SM.  Whatever
+    the cost model prefers, the parts must tile the pairs exactly, in order, on no more CTAs than SMs; no row tile may be
+    touched by more parts than the eight-bit arrival count of an accumulate word can hold; and the split must be the
+    same every time (the plan is cached)."""
+    lib = ctypes.CDLL(rabit.lib_path())
+    lib.rabit_selftest_f16_plan.restype = ctypes.c_int
+    lib.rabit_selftest_f16_plan.argtypes = [ctypes.c_int] * 5 + [ctypes.c_void_p, ctypes.c_int]
+    out = (ctypes.c_int * 400)()
+    grid = lib.rabit_selftest_f16_plan(K, M, N, batch, sms, out, 400)
+    n_rt, n_cs = -(-M // 128), -(-N // 256)
+    n_pairs = n_rt * n_cs
+    assert 1 <= grid <= min(sms, n_pairs)
+    bound = list(out[:2 * grid + 1])
+    assert bound[0] == 0 and bound[-1] == n_pairs
+    assert all(a <= b for a, b in zip(bound, bound[1:]))
+    parts = [(a, b) for a, b in zip(bound, bound[1:]) if b > a]
+    assert sum(b - a for a, b in parts) == n_pairs
+    assert all(bound[2 * c] < bound[2 * c + 2] for c in range(grid))             # every CTA has work
+    touching = [0] * n_rt
+    for a, b in parts:
+        for rt in range(a // n_cs, (b - 1) // n_cs + 1):
+            touching[rt] += 1
+    assert 1 <= min(touching) and max(touching) <= 255
+    # balance: no SM has more than twice the average number of pairs (plus one row tile's worth of slack for tiny layers)
+    per_sm = [bound[2 * c + 2] - bound[2 * c] for c in range(grid)]
+    assert max(per_sm) <= 2 * n_pairs / grid + n_cs
+    again = (ctypes.c_int * 400)()
+    assert lib.rabit_selftest_f16_plan(K, M, N, batch, sms, again, 400) == grid and list(again[:2 * grid + 1]) == bound
+
+
+def test_work_split_of_the_f16_gemv_rejects_what_the_kernel_cannot_run():
+    lib = ctypes.CDLL(rabit.lib_path())
+    lib.rabit_selftest_f16_plan.restype = ctypes.c_int
+    lib.rabit_selftest_f16_plan.argtypes = [ctypes.c_int] * 5 + [ctypes.c_void_p, ctypes.c_int]
+    out = (ctypes.c_int * 400)()
+    assert lib.rabit_selftest_f16_plan(2, 128, 65312, 8, 148, out, 400) < 0      # 256 slices
+    assert lib.rabit_selftest_f16_plan(2, 128, 4096, 17, 148, out, 400) < 0      # more rows than a pass takes
+    assert lib.rabit_selftest_f16_plan(4, 128, 4096, 8, 148, out, 400) < 0       # too many paths
+    assert lib.rabit_selftest_f16_plan(2, 4096, 4096, 8, 148, out, 10) < 0       # output array too small
+    assert lib.rabit_selftest_f16_plan(2, 4096, 4096, 8, 148, None, 400) < 0
